@@ -1,0 +1,178 @@
+/*
+ * keydiff.h -- C ABI of the B200 (sm_100a) KeyDiff eviction-step library.
+ *
+ * The library implements one operation: the per-KV-head cache eviction step of
+ * KeyDiff's block-wise prefill (Sec. 2.3-2.4 and 3.2 of the paper).  After a block of
+ * B new keys/values is appended to a cache bounded by a budget of N tokens, every
+ * (layer, sequence, KV head) unit independently
+ *   1. forms the anchor  mu = (1/n) sum_i k_i/||k_i||  over its n = len + B keys,
+ *   2. scores each key   s_i = mu.k_i / max(||mu||*||k_i||, eps)        (App. B.1),
+ *   3. keeps the N keys with the LOWEST cosine (Eq. efficient-keydiff:
+ *      S = topk(-CosSim(mu, k_i), N)), ties keeping the older token,
+ *   4. gathers K' = gather(K,S), V' = gather(V,S) (Eq. keydiff) in original token
+ *      order, in place.
+ *
+ * Conventions
+ *   - No exceptions cross this boundary.  Every call returns an int status
+ *     (KEYDIFF_OK or a negative KEYDIFF_ERR_*); keydiff_strerror names it.
+ *   - "device" pointers are CUDA global-memory addresses on the ctx's device;
+ *     "host" pointers are ordinary process memory.
+ *   - All work is enqueued on the given stream; nothing here synchronises with the
+ *     host unless stated.  keydiff_evict allocates nothing.
+ *   - Not thread-safe per ctx: use a ctx from one host thread / one stream at a
+ *     time.  Distinct ctxs are independent.
+ *   - There is no CPU fallback: on a machine without a usable sm_100 device
+ *     keydiff_create fails with KEYDIFF_ERR_CUDA / KEYDIFF_ERR_UNSUPPORTED.
+ *
+ * Tensor layouts (bf16, contiguous, row = token):
+ *   k_cache, v_cache : [n_layers][batch][n_kv_heads][budget N][head_dim]
+ *                      rows [0, len) of every unit are valid
+ *   new_k,  new_v    : [n_layers][batch][n_kv_heads][block B][head_dim]
+ *   All four base pointers must be 16-byte aligned.  The caches and the blocks
+ *   must not overlap.
+ */
+#ifndef KEYDIFF_H_
+#define KEYDIFF_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define KEYDIFF_API __attribute__((visibility("default")))
+#else
+#define KEYDIFF_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct keydiff_ctx keydiff_ctx; /* opaque; owns only its scratch memory */
+
+enum {
+    KEYDIFF_OK = 0,
+    KEYDIFF_ERR_INVALID_ARG = -1, /* NULL / misaligned pointer, value out of range, mismatch with ctx */
+    KEYDIFF_ERR_UNSUPPORTED = -2, /* valid request this build cannot serve (dtype, head_dim, size, device) */
+    KEYDIFF_ERR_ALLOC = -3,       /* scratch allocation failed in keydiff_create */
+    KEYDIFF_ERR_CUDA = -4,        /* a CUDA runtime call failed; see keydiff_last_cuda_error */
+    KEYDIFF_ERR_STATE = -5,       /* call not valid in the ctx's current state */
+    KEYDIFF_ERR_TIMEOUT = -6      /* a bounded device-side wait expired (reported in the status word) */
+};
+
+enum { KEYDIFF_BF16 = 0 };
+
+/* Which kernels serve keydiff_evict. */
+enum {
+    KEYDIFF_PATH_AUTO = 0,    /* fused cluster kernel when a unit fits, else the staged kernels */
+    KEYDIFF_PATH_STAGED = 1,  /* four launches: anchor partials, scores, select, compaction */
+    KEYDIFF_PATH_FUSED = 2    /* one launch, one thread-block cluster per unit; create fails
+                                 with KEYDIFF_ERR_UNSUPPORTED if a unit cannot fit */
+};
+
+typedef struct {
+    int32_t n_layers;      /* >= 1 */
+    int32_t batch;         /* >= 1, independent sequences */
+    int32_t n_kv_heads;    /* >= 1, KV heads per layer (GQA groups share one KV head) */
+    int32_t head_dim;      /* 128 (the only value built) */
+    int32_t budget;        /* N, cache budget in tokens (Sec. 2.3), >= 1 */
+    int32_t max_block;     /* largest B ever passed to keydiff_evict (Sec. 2.4), >= 1 */
+    int32_t dtype;         /* KEYDIFF_BF16 */
+    int32_t path;          /* KEYDIFF_PATH_* */
+    float   eps;           /* eps of App. B.1's max(.,eps); 0 selects the default 1e-8 */
+    int32_t device;        /* CUDA device ordinal */
+} keydiff_config;
+
+/*
+ * keydiff_create -- allocate a context and its device scratch for U = n_layers*batch*
+ * n_kv_heads units (scores U*(N+max_block) fp32, kept-index list U*N int32, anchor
+ * partials, per-unit counters, one status word).  Synchronous.  *out is set only on
+ * KEYDIFF_OK.  The initial cache length is 0 (C_0 = empty, Eq. block_processing).
+ * Errors: INVALID_ARG (NULL, non-positive sizes), UNSUPPORTED (dtype, head_dim, a unit
+ * too large for the requested path, no sm_100 device), ALLOC, CUDA.
+ */
+KEYDIFF_API int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out);
+
+/*
+ * keydiff_evict -- one step of Eq. (block_processing) for every unit of the ctx:
+ * C <- ([K || new_k], [V || new_v]); C <- pi_N(C) with pi_N = KeyDiff (Eq.
+ * efficient-keydiff, anchor of normalised keys).
+ *   n = len + block_B.  If n <= N the block rows are appended at rows [len, n) and
+ *   nothing is scored (Sec. 2.3: eviction only when the budget is exceeded).
+ *   Otherwise the n keys are scored, the N with the largest eviction score e = -s are
+ *   kept (ties: lower token index wins), and K and V are compacted in place in
+ *   original token order; rows in front of the first evicted row are not touched.
+ *   Afterwards len = min(N, n) for every unit.
+ * k_cache, v_cache: device, in/out, caller-owned.  new_k, new_v: device, read only,
+ * caller-owned; they may be reused once the work enqueued on `stream` has completed.
+ * budget_N, n_kv_heads, head_dim restate the ctx's values and must equal them;
+ * 1 <= block_B <= max_block.  stream: a cudaStream_t (NULL = legacy default stream).
+ * Asynchronous: returns after enqueueing.  Host-detectable errors (INVALID_ARG,
+ * STATE) enqueue nothing and leave len unchanged.  Device-side anomalies (a bounded
+ * wait that expired) are written to the status word (keydiff_get_scratch) and the
+ * kernels return normally.  Non-finite keys give an unspecified selection, never a
+ * fault.
+ */
+KEYDIFF_API int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache,
+                  const void* new_k, const void* new_v,
+                  int32_t budget_N, int32_t block_B, int32_t n_kv_heads, int32_t head_dim,
+                  void* stream);
+
+/*
+ * keydiff_evict_host -- the same step with the BLOCK in host memory (the caches stay on
+ * the device): copies new_k/new_v (host, block_B rows per unit, same layout) to ctx-owned
+ * device staging on `stream`, runs keydiff_evict, then copies the kept-index list
+ * (U*N int32, see keydiff_get_scratch) and the status word back into kept_idx_host /
+ * status_host (host; either may be NULL to skip).  Pinned host memory makes the copies
+ * asynchronous; the call itself does not synchronise.  The staging buffers are allocated
+ * on first use (that first call synchronises and may return ALLOC).
+ */
+KEYDIFF_API int keydiff_evict_host(keydiff_ctx* ctx, void* k_cache, void* v_cache,
+                       const void* new_k_host, const void* new_v_host,
+                       int32_t budget_N, int32_t block_B, int32_t n_kv_heads, int32_t head_dim,
+                       int32_t* kept_idx_host, int32_t* status_host, void* stream);
+
+/* keydiff_destroy -- free the scratch and the ctx.  Synchronises the device.  NULL is OK. */
+KEYDIFF_API int keydiff_destroy(keydiff_ctx* ctx);
+
+/* Cache length bookkeeping (host side, no device work).  C_0 = empty: reset sets len = 0;
+ * set_len resumes from a cache the caller restored (0 <= len <= N). */
+KEYDIFF_API int keydiff_reset(keydiff_ctx* ctx);
+KEYDIFF_API int keydiff_get_len(const keydiff_ctx* ctx, int32_t* len_out);
+KEYDIFF_API int keydiff_set_len(keydiff_ctx* ctx, int32_t len);
+
+/*
+ * keydiff_get_scratch -- device pointers into ctx-owned scratch, valid until destroy;
+ * contents are those of the most recent evicting step once its stream work completed.
+ *   scores   : [U][N + max_block] fp32, e_i = -s_i for i < n (the eviction score, +0 for -0)
+ *   kept_idx : [U][N] int32, ascending token indices (into the n concatenated rows) of
+ *              the kept tokens = source row of every destination row
+ *   first_evicted : [U] int32, index of the first evicted token (rows before it did not move)
+ *   status   : [1] int32, 0 or a KEYDIFF_ERR_* code set by a kernel
+ * Any output pointer may be NULL.
+ */
+KEYDIFF_API int keydiff_get_scratch(const keydiff_ctx* ctx, const float** scores, const int32_t** kept_idx,
+                        const int32_t** first_evicted, const int32_t** status);
+
+/*
+ * keydiff_get_moved_rows -- device pointer to a 64-bit counter: the number of kept rows (per
+ * tensor) whose position changed, summed over all units and all evicting steps since create
+ * (= sum over units of N - first_evicted).  Benchmarks use it to count the bytes a step had to
+ * move.  Read it after synchronising the stream.
+ */
+KEYDIFF_API int keydiff_get_moved_rows(const keydiff_ctx* ctx, const unsigned long long** counter);
+
+/* Launch facts of the chosen path, for benchmarks: path actually used (KEYDIFF_PATH_*),
+ * kernels launched per evicting step, cluster size (1 for the staged path). */
+KEYDIFF_API int keydiff_get_launch_info(const keydiff_ctx* ctx, int32_t* path, int32_t* launches_per_step,
+                            int32_t* cluster_size);
+
+/* Text of a status code; never NULL. */
+KEYDIFF_API const char* keydiff_strerror(int code);
+
+/* cudaError_t value of the most recent failed CUDA call made by this library on the
+ * calling thread (0 if none). */
+KEYDIFF_API int keydiff_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KEYDIFF_H_ */

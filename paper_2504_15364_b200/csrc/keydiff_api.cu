@@ -1,0 +1,283 @@
+// Host side of the KeyDiff eviction-step library: context, argument validation, launch
+// configuration and the extern "C" entry points declared in include/keydiff.h.
+#include "../../include/keydiff.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <new>
+
+#include "common.cuh"
+#include "staged_kernels.cuh"
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+inline bool cuda_ok(cudaError_t e) {
+    if (e == cudaSuccess) return true;
+    g_last_cuda_error = static_cast<int>(e);
+    return false;
+}
+#define KD_CUDA(call) do { if (!cuda_ok(call)) return KEYDIFF_ERR_CUDA; } while (0)
+
+constexpr float kDefaultEps = 1e-8f;
+constexpr int kMaxSelectSmem = 200 * 1024;   // score keys of one unit must fit one CTA
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+struct keydiff_ctx {
+    keydiff_config cfg;
+    int U = 0;            // independent units = n_layers * batch * n_kv_heads
+    int nmax = 0;         // N + max_block
+    int len = 0;          // tokens currently cached (same for every unit)
+    int splits = 1;       // row slices per unit in the staged anchor/score kernels
+    int path = KEYDIFF_PATH_STAGED;
+    int cluster = 1;
+    float eps = kDefaultEps;
+    // device scratch
+    float* partial = nullptr;         // [U][splits][128]
+    float* norms = nullptr;           // [U][nmax]
+    float* scores = nullptr;          // [U][nmax]
+    int32_t* kept_idx = nullptr;      // [U][N]
+    int32_t* first_evicted = nullptr; // [U]
+    int32_t* status = nullptr;        // [1]
+    unsigned long long* moved_rows = nullptr;   // [1] cumulative count of rows that changed position
+    void* stage_k = nullptr;          // [U][max_block][128] bf16, keydiff_evict_host only
+    void* stage_v = nullptr;
+};
+
+namespace {
+
+void free_scratch(keydiff_ctx* c) {
+    cudaFree(c->partial); cudaFree(c->norms); cudaFree(c->scores); cudaFree(c->kept_idx);
+    cudaFree(c->first_evicted); cudaFree(c->status); cudaFree(c->moved_rows); cudaFree(c->stage_k); cudaFree(c->stage_v);
+}
+
+int check_step_args(const keydiff_ctx* ctx, const void* k_cache, const void* v_cache,
+                    const void* new_k, const void* new_v, int32_t N, int32_t B, int32_t H, int32_t d) {
+    if (!ctx || !k_cache || !v_cache || !new_k || !new_v) return KEYDIFF_ERR_INVALID_ARG;
+    if (N != ctx->cfg.budget || H != ctx->cfg.n_kv_heads || d != ctx->cfg.head_dim) return KEYDIFF_ERR_INVALID_ARG;
+    if (B < 1 || B > ctx->cfg.max_block) return KEYDIFF_ERR_INVALID_ARG;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(new_k) || !aligned16(new_v)) return KEYDIFF_ERR_INVALID_ARG;
+    if (k_cache == v_cache || k_cache == new_k || v_cache == new_v) return KEYDIFF_ERR_INVALID_ARG;
+    int dev = -1;
+    KD_CUDA(cudaGetDevice(&dev));
+    if (dev != ctx->cfg.device) return KEYDIFF_ERR_STATE;   // the ctx's device must be current
+    return KEYDIFF_OK;
+}
+
+int launch_staged(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const uint4* nv, int B, cudaStream_t st) {
+    using namespace kd;
+    const int N = c->cfg.budget, n = c->len + B, U = c->U;
+    const int rows_per_split = (n + c->splits - 1) / c->splits;
+    const dim3 grid(c->splits, U);
+    anchor_partial_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, c->len, B, N, c->eps, rows_per_split, c->nmax,
+                                                           c->partial, c->norms);
+    score_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, c->len, B, N, c->eps, rows_per_split, c->nmax,
+                                                  c->partial, c->norms, c->scores);
+    select_kernel<<<U, kSelectThreads, static_cast<size_t>(n) * 4, st>>>(c->scores, n, N, c->nmax, c->len, c->kept_idx,
+                                                                          c->first_evicted, c->moved_rows);
+    compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, c->len, B, N, c->kept_idx, c->first_evicted);
+    KD_CUDA(cudaGetLastError());
+    return KEYDIFF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
+    if (!cfg || !out) return KEYDIFF_ERR_INVALID_ARG;
+    if (cfg->n_layers < 1 || cfg->batch < 1 || cfg->n_kv_heads < 1 || cfg->budget < 1 || cfg->max_block < 1 ||
+        cfg->device < 0 || cfg->eps < 0.f)
+        return KEYDIFF_ERR_INVALID_ARG;
+    if (cfg->path != KEYDIFF_PATH_AUTO && cfg->path != KEYDIFF_PATH_STAGED && cfg->path != KEYDIFF_PATH_FUSED)
+        return KEYDIFF_ERR_INVALID_ARG;
+    if (cfg->dtype != KEYDIFF_BF16 || cfg->head_dim != kd::kHeadDim) return KEYDIFF_ERR_UNSUPPORTED;
+    const long long U = 1LL * cfg->n_layers * cfg->batch * cfg->n_kv_heads;
+    const long long nmax = 1LL * cfg->budget + cfg->max_block;
+    if (U > 65535 || nmax > (1 << 30)) return KEYDIFF_ERR_UNSUPPORTED;   // gridDim.y limit of the staged kernels
+    if (nmax * 4 > kMaxSelectSmem) return KEYDIFF_ERR_UNSUPPORTED;
+    if (cfg->path == KEYDIFF_PATH_FUSED) return KEYDIFF_ERR_UNSUPPORTED;
+
+    int count = 0;
+    KD_CUDA(cudaGetDeviceCount(&count));
+    if (cfg->device >= count) return KEYDIFF_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    KD_CUDA(cudaGetDeviceProperties(&prop, cfg->device));
+    if (prop.major != 10) return KEYDIFF_ERR_UNSUPPORTED;   // built for sm_100a only; no fallback
+
+    int prev = -1;
+    KD_CUDA(cudaGetDevice(&prev));
+    KD_CUDA(cudaSetDevice(cfg->device));
+
+    keydiff_ctx* c = new (std::nothrow) keydiff_ctx();
+    if (!c) { cudaSetDevice(prev); return KEYDIFF_ERR_ALLOC; }
+    c->cfg = *cfg;
+    c->U = static_cast<int>(U);
+    c->nmax = static_cast<int>(nmax);
+    c->eps = cfg->eps > 0.f ? cfg->eps : kDefaultEps;
+    c->path = KEYDIFF_PATH_STAGED;
+    // enough CTAs to fill 148 SMs a few times over, but at least 64 rows per slice
+    const int want = (4 * prop.multiProcessorCount + c->U - 1) / c->U;
+    c->splits = std::max(1, std::min({want, (c->nmax + 63) / 64, 64}));
+
+    bool ok = true;
+    ok = ok && cudaMalloc(&c->partial, sizeof(float) * c->U * c->splits * kd::kHeadDim) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->norms, sizeof(float) * U * nmax) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->scores, sizeof(float) * U * nmax) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->kept_idx, sizeof(int32_t) * U * cfg->budget) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->first_evicted, sizeof(int32_t) * U) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->status, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->moved_rows, sizeof(unsigned long long)) == cudaSuccess;
+    if (ok) {
+        ok = cudaMemset(c->scores, 0, sizeof(float) * U * nmax) == cudaSuccess &&
+             cudaMemset(c->kept_idx, 0, sizeof(int32_t) * U * cfg->budget) == cudaSuccess &&
+             cudaMemset(c->first_evicted, 0, sizeof(int32_t) * U) == cudaSuccess &&
+             cudaMemset(c->status, 0, sizeof(int32_t)) == cudaSuccess &&
+             cudaMemset(c->moved_rows, 0, sizeof(unsigned long long)) == cudaSuccess;
+    }
+    if (ok) {
+        ok = cudaFuncSetAttribute(kd::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  kMaxSelectSmem) == cudaSuccess;
+    }
+    if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) {
+        g_last_cuda_error = static_cast<int>(cudaGetLastError());
+        free_scratch(c);
+        delete c;
+        cudaSetDevice(prev);
+        return KEYDIFF_ERR_ALLOC;
+    }
+    cudaSetDevice(prev);
+    *out = c;
+    return KEYDIFF_OK;
+}
+
+int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache, const void* new_k, const void* new_v,
+                  int32_t budget_N, int32_t block_B, int32_t n_kv_heads, int32_t head_dim, void* stream) {
+    const int rc = check_step_args(ctx, k_cache, v_cache, new_k, new_v, budget_N, block_B, n_kv_heads, head_dim);
+    if (rc != KEYDIFF_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint4* kc = static_cast<uint4*>(k_cache);
+    uint4* vc = static_cast<uint4*>(v_cache);
+    const uint4* nk = static_cast<const uint4*>(new_k);
+    const uint4* nv = static_cast<const uint4*>(new_v);
+    const int N = ctx->cfg.budget, n = ctx->len + block_B;
+    if (n <= N) {
+        // Sec. 2.3: the budget is not exceeded, nothing is evicted
+        const int threads = 256;
+        const dim3 grid((block_B * kd::kRowVec + threads - 1) / threads, ctx->U, 2);
+        kd::append_kernel<<<grid, threads, 0, st>>>(kc, vc, nk, nv, ctx->len, block_B, N);
+        KD_CUDA(cudaGetLastError());
+        ctx->len = n;
+        return KEYDIFF_OK;
+    }
+    const int lrc = launch_staged(ctx, kc, vc, nk, nv, block_B, st);
+    if (lrc != KEYDIFF_OK) return lrc;
+    ctx->len = N;
+    return KEYDIFF_OK;
+}
+
+int keydiff_evict_host(keydiff_ctx* ctx, void* k_cache, void* v_cache, const void* new_k_host, const void* new_v_host,
+                       int32_t budget_N, int32_t block_B, int32_t n_kv_heads, int32_t head_dim,
+                       int32_t* kept_idx_host, int32_t* status_host, void* stream) {
+    if (!ctx || !new_k_host || !new_v_host) return KEYDIFF_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!ctx->stage_k) {
+        const size_t bytes = static_cast<size_t>(ctx->U) * ctx->cfg.max_block * kd::kRowBytes;
+        if (cudaMalloc(&ctx->stage_k, bytes) != cudaSuccess || cudaMalloc(&ctx->stage_v, bytes) != cudaSuccess) {
+            g_last_cuda_error = static_cast<int>(cudaGetLastError());
+            cudaFree(ctx->stage_k); ctx->stage_k = nullptr;
+            return KEYDIFF_ERR_ALLOC;
+        }
+    }
+    const int rc = check_step_args(ctx, k_cache, v_cache, ctx->stage_k, ctx->stage_v, budget_N, block_B, n_kv_heads, head_dim);
+    if (rc != KEYDIFF_OK) return rc;
+    const size_t bytes = static_cast<size_t>(ctx->U) * block_B * kd::kRowBytes;
+    KD_CUDA(cudaMemcpyAsync(ctx->stage_k, new_k_host, bytes, cudaMemcpyHostToDevice, st));
+    KD_CUDA(cudaMemcpyAsync(ctx->stage_v, new_v_host, bytes, cudaMemcpyHostToDevice, st));
+    const int erc = keydiff_evict(ctx, k_cache, v_cache, ctx->stage_k, ctx->stage_v, budget_N, block_B, n_kv_heads,
+                                  head_dim, stream);
+    if (erc != KEYDIFF_OK) return erc;
+    if (kept_idx_host)
+        KD_CUDA(cudaMemcpyAsync(kept_idx_host, ctx->kept_idx, sizeof(int32_t) * ctx->U * ctx->cfg.budget,
+                                cudaMemcpyDeviceToHost, st));
+    if (status_host)
+        KD_CUDA(cudaMemcpyAsync(status_host, ctx->status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    return KEYDIFF_OK;
+}
+
+int keydiff_destroy(keydiff_ctx* ctx) {
+    if (!ctx) return KEYDIFF_OK;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    cudaSetDevice(ctx->cfg.device);
+    cudaDeviceSynchronize();
+    free_scratch(ctx);
+    if (prev >= 0) cudaSetDevice(prev);
+    delete ctx;
+    return KEYDIFF_OK;
+}
+
+int keydiff_reset(keydiff_ctx* ctx) {
+    if (!ctx) return KEYDIFF_ERR_INVALID_ARG;
+    ctx->len = 0;
+    return KEYDIFF_OK;
+}
+
+int keydiff_get_len(const keydiff_ctx* ctx, int32_t* len_out) {
+    if (!ctx || !len_out) return KEYDIFF_ERR_INVALID_ARG;
+    *len_out = ctx->len;
+    return KEYDIFF_OK;
+}
+
+int keydiff_set_len(keydiff_ctx* ctx, int32_t len) {
+    if (!ctx || len < 0 || len > ctx->cfg.budget) return KEYDIFF_ERR_INVALID_ARG;
+    ctx->len = len;
+    return KEYDIFF_OK;
+}
+
+int keydiff_get_scratch(const keydiff_ctx* ctx, const float** scores, const int32_t** kept_idx,
+                        const int32_t** first_evicted, const int32_t** status) {
+    if (!ctx) return KEYDIFF_ERR_INVALID_ARG;
+    if (scores) *scores = ctx->scores;
+    if (kept_idx) *kept_idx = ctx->kept_idx;
+    if (first_evicted) *first_evicted = ctx->first_evicted;
+    if (status) *status = ctx->status;
+    return KEYDIFF_OK;
+}
+
+int keydiff_get_moved_rows(const keydiff_ctx* ctx, const unsigned long long** counter) {
+    if (!ctx || !counter) return KEYDIFF_ERR_INVALID_ARG;
+    *counter = ctx->moved_rows;
+    return KEYDIFF_OK;
+}
+
+int keydiff_get_launch_info(const keydiff_ctx* ctx, int32_t* path, int32_t* launches_per_step, int32_t* cluster_size) {
+    if (!ctx) return KEYDIFF_ERR_INVALID_ARG;
+    if (path) *path = ctx->path;
+    if (launches_per_step) *launches_per_step = ctx->path == KEYDIFF_PATH_FUSED ? 1 : 4;
+    if (cluster_size) *cluster_size = ctx->cluster;
+    return KEYDIFF_OK;
+}
+
+const char* keydiff_strerror(int code) {
+    switch (code) {
+        case KEYDIFF_OK: return "ok";
+        case KEYDIFF_ERR_INVALID_ARG: return "invalid argument";
+        case KEYDIFF_ERR_UNSUPPORTED: return "unsupported configuration or device";
+        case KEYDIFF_ERR_ALLOC: return "device memory allocation failed";
+        case KEYDIFF_ERR_CUDA: return "CUDA runtime error";
+        case KEYDIFF_ERR_STATE: return "call not valid in the current state (is the ctx's device current?)";
+        case KEYDIFF_ERR_TIMEOUT: return "bounded device-side wait expired";
+        default: return "unknown keydiff status";
+    }
+}
+
+int keydiff_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"
