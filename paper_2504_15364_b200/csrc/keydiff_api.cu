@@ -9,6 +9,7 @@
 
 #include "common.cuh"
 #include "staged_kernels.cuh"
+#include "fused_kernel.cuh"
 
 namespace {
 
@@ -35,7 +36,11 @@ struct keydiff_ctx {
     int len = 0;          // tokens currently cached (same for every unit)
     int splits = 1;       // row slices per unit in the staged anchor/score kernels
     int path = KEYDIFF_PATH_STAGED;
-    int cluster = 1;
+    int cluster = 1;            // fused path: CTAs per cluster
+    int fused_smem_rows = 0;    // fused path: slice rows resident in shared memory
+    int fused_nkeys = 0;        // fused path: key-table capacity
+    int fused_smem_bytes = 0;
+    int fused_max_clusters = 0; // co-resident clusters (grid = min(U, this) * cluster)
     float eps = kDefaultEps;
     // device scratch
     float* partial = nullptr;         // [U][splits][128]
@@ -66,6 +71,74 @@ int check_step_args(const keydiff_ctx* ctx, const void* k_cache, const void* v_c
     int dev = -1;
     KD_CUDA(cudaGetDevice(&dev));
     if (dev != ctx->cfg.device) return KEYDIFF_ERR_STATE;   // the ctx's device must be current
+    return KEYDIFF_OK;
+}
+
+// Choose the cluster size and shared-memory split of the fused kernel for units of up to nmax
+// rows; returns false if no cluster can hold a unit on chip.
+bool plan_fused(keydiff_ctx* c, int sm_count) {
+    using namespace kd;
+    const int nkeys = (c->nmax + 31) & ~31;
+    int chosen = 0, chosen_rows = 0;
+    for (int C = 1; C <= 16; C *= 2) {
+        const int per_cta = (c->nmax + C - 1) / C;
+        int sr = kMaxChunks * kChunkRows;
+        while (sr > 0 && fused_layout(sr, nkeys).total > kSmemLimit) sr -= kChunkRows;
+        if (sr <= 0) return false;                                   // the key table alone does not fit
+        if (sr + kRegRows * kGroups < per_cta) continue;             // slice too long for this cluster size
+        // small jobs: spread a unit over more SMs while the whole grid still fits the device
+        if (chosen == 0 || (C <= 8 && c->U * C <= sm_count)) {
+            chosen = C;
+            chosen_rows = std::min(sr, (per_cta + kChunkRows - 1) / kChunkRows * kChunkRows);
+        }
+        if (C * 2 > 8 && chosen != 0) break;
+    }
+    if (chosen == 0) return false;
+    const FusedLayout L = fused_layout(chosen_rows, nkeys);
+    if (cudaFuncSetAttribute(fused_evict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess) return false;
+    if (chosen > 8 &&
+        cudaFuncSetAttribute(fused_evict_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return false;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(chosen * sm_count);
+    cfg.blockDim = dim3(kFusedThreads);
+    cfg.dynamicSmemBytes = L.total;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = chosen; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int max_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, fused_evict_kernel, &cfg) != cudaSuccess || max_clusters < 1) {
+        cudaGetLastError();
+        return false;
+    }
+    c->cluster = chosen;
+    c->fused_smem_rows = chosen_rows;
+    c->fused_nkeys = nkeys;
+    c->fused_smem_bytes = L.total;
+    c->fused_max_clusters = max_clusters;
+    return true;
+}
+
+int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const uint4* nv, int B, cudaStream_t st) {
+    using namespace kd;
+    FusedParams p;
+    p.k_cache = kc; p.v_cache = vc; p.new_k = nk; p.new_v = nv;
+    p.len = c->len; p.B = B; p.N = c->cfg.budget; p.U = c->U; p.eps = c->eps;
+    p.cluster = c->cluster;
+    p.rows_per_cta = (c->len + B + c->cluster - 1) / c->cluster;
+    p.smem_rows = c->fused_smem_rows; p.nkeys = c->fused_nkeys; p.nmax = c->nmax;
+    p.scores = c->scores; p.kept_idx = c->kept_idx; p.first_evicted = c->first_evicted;
+    p.moved_rows = c->moved_rows; p.status = c->status;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(std::min(c->U, c->fused_max_clusters) * c->cluster);
+    cfg.blockDim = dim3(kFusedThreads);
+    cfg.dynamicSmemBytes = c->fused_smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = c->cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    KD_CUDA(cudaLaunchKernelEx(&cfg, fused_evict_kernel, p));
     return KEYDIFF_OK;
 }
 
@@ -101,7 +174,6 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
     const long long nmax = 1LL * cfg->budget + cfg->max_block;
     if (U > 65535 || nmax > (1 << 30)) return KEYDIFF_ERR_UNSUPPORTED;   // gridDim.y limit of the staged kernels
     if (nmax * 4 > kMaxSelectSmem) return KEYDIFF_ERR_UNSUPPORTED;
-    if (cfg->path == KEYDIFF_PATH_FUSED) return KEYDIFF_ERR_UNSUPPORTED;
 
     int count = 0;
     KD_CUDA(cudaGetDeviceCount(&count));
@@ -145,6 +217,16 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
                                   kMaxSelectSmem) == cudaSuccess;
     }
     if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
+    if (ok && cfg->path != KEYDIFF_PATH_STAGED) {
+        if (plan_fused(c, prop.multiProcessorCount)) {
+            c->path = KEYDIFF_PATH_FUSED;
+        } else if (cfg->path == KEYDIFF_PATH_FUSED) {
+            free_scratch(c);
+            delete c;
+            cudaSetDevice(prev);
+            return KEYDIFF_ERR_UNSUPPORTED;
+        }
+    }
     if (!ok) {
         g_last_cuda_error = static_cast<int>(cudaGetLastError());
         free_scratch(c);
@@ -176,7 +258,8 @@ int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache, const void* ne
         ctx->len = n;
         return KEYDIFF_OK;
     }
-    const int lrc = launch_staged(ctx, kc, vc, nk, nv, block_B, st);
+    const int lrc = ctx->path == KEYDIFF_PATH_FUSED ? launch_fused(ctx, kc, vc, nk, nv, block_B, st)
+                                                    : launch_staged(ctx, kc, vc, nk, nv, block_B, st);
     if (lrc != KEYDIFF_OK) return lrc;
     ctx->len = N;
     return KEYDIFF_OK;

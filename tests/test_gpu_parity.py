@@ -12,7 +12,7 @@ from paper_2504_15364_b200 import KeyDiff, KeyDiffError, binding, synth
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-PATHS = [binding.KEYDIFF_PATH_STAGED]
+PATHS = [binding.KEYDIFF_PATH_STAGED, binding.KEYDIFF_PATH_FUSED]
 
 
 def bits(t: torch.Tensor) -> np.ndarray:
