@@ -1,0 +1,289 @@
+#!/usr/bin/env python
+"""Benchmark of the KeyDiff eviction step (steps/s and achieved HBM bandwidth).
+
+A step is one ``keydiff_evict`` call over all units of the workload for one appended block, in
+steady state (cache at its budget, B rows evicted per unit).  Default workload: the
+Llama-3.1-8B-shaped config (32 layers x 8 KV heads, N=8192, B=128, 32K-token prompt).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--path auto|staged|fused]
+  python bench.py --impl reference ...        # the CPU oracle on the host cores, same metric
+
+Prints ONE JSON line (rank 0).  Under torchrun every rank runs its own replica of the workload
+(different seeded sequences); ``value`` is the whole-job rate against the slowest rank.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2504_15364_b200 import synth
+from paper_2504_15364_b200 import dist as kdist
+
+METRIC = "eviction_steps_per_s"
+UNIT = "steps/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (bytes per step of the named workload); None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def algorithmic_bytes(wl, moved_rows_per_step_per_unit: float) -> float:
+    """Bytes one evicting step must move: every key read once, moved K rows written, moved V rows
+    read and written, fp32 scores written once and read once."""
+    row = wl.head_dim * 2
+    n = wl.budget + wl.block
+    per_unit = n * row + 3.0 * moved_rows_per_step_per_unit * row + 2 * n * 4
+    return wl.units * per_unit
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock, power and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.stop_flag = index, [], set(), False
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                break
+            time.sleep(0.002)
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def bits(t):
+    return t.detach().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def run_ours(args):
+    from paper_2504_15364_b200 import KeyDiff, binding
+    rank, world, local = kdist.init_from_env()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    wl = synth.WORKLOADS[args.workload]
+    U, N, B, d = wl.units, wl.budget, wl.block, wl.head_dim
+    path = {"auto": binding.KEYDIFF_PATH_AUTO, "staged": binding.KEYDIFF_PATH_STAGED,
+            "fused": binding.KEYDIFF_PATH_FUSED}[args.path]
+    K, W = args.steps, args.warmup
+    K2 = 0 if args.no_e2e else min(K, 40)
+
+    stream = synth.KVStream(wl, dev, rank=rank)
+    k_cache = torch.zeros(U, N, d, dtype=torch.bfloat16, device=dev)
+    v_cache = torch.zeros_like(k_cache)
+    kd = KeyDiff(wl.n_layers, wl.batch, wl.n_kv_heads, d, N, B, path=path, device=local)
+    info = kd.launch_info()
+    # fill through the library's append path (C_0 = empty)
+    for _ in range(wl.fill_steps):
+        nk, nv = stream.next_block()
+        kd.evict(k_cache, v_cache, nk, nv)
+    assert kd.len == N
+    blocks = [stream.next_block() for _ in range(W + K)]
+    torch.cuda.synchronize()
+
+    for i in range(W):
+        kd.evict(k_cache, v_cache, *blocks[i])
+    torch.cuda.synchronize()
+    moved0 = kd.moved_rows()
+
+    st = torch.cuda.current_stream(dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    sampler = ClockSampler(local)
+    kdist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev[0].record(st)
+    for i in range(K):
+        kd.evict(k_cache, v_cache, *blocks[W + i])
+        ev[i + 1].record(st)
+    torch.cuda.synchronize()
+    sampler.stop_flag = True
+    kdist.barrier()
+    sampler.join()
+    total_ms = ev[0].elapsed_time(ev[K])
+    step_ms = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(K)])
+    moved = (kd.moved_rows() - moved0) / K / U
+    status = int(kd.scratch()["status"].item())
+    assert status == 0, f"device status {status}"
+
+    total_ms_max = kdist.max_over_ranks(total_ms, dev)
+    steps_total = kdist.sum_over_ranks(K, dev)
+    value = steps_total / (total_ms_max * 1e-3)
+
+    # ---- end to end: block from pinned host memory, kept-index list + status read back
+    e2e = None
+    if K2:
+        host_blocks = [tuple(t.cpu().pin_memory() for t in stream.next_block()) for _ in range(K2 + 2)]
+        kept_h = torch.empty(U, N, dtype=torch.int32).pin_memory()
+        status_h = torch.zeros(1, dtype=torch.int32).pin_memory()
+        for i in range(2):
+            kd.evict_host(k_cache, v_cache, *host_blocks[i], kept_h, status_h)
+        kdist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for i in range(K2):
+            kd.evict_host(k_cache, v_cache, *host_blocks[2 + i], kept_h, status_h)
+        e1.record(st)
+        torch.cuda.synchronize()
+        kdist.barrier()
+        e2e_ms = kdist.max_over_ranks(e0.elapsed_time(e1), dev)
+        e2e = {"value": kdist.sum_over_ranks(K2, dev) / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": 2 * U * B * d * 2, "d2h_bytes_per_step": U * N * 4 + 4, "steps": K2}
+
+    if rank != 0:
+        return
+    peak, peak_src = measured_peak()
+    a_step = algorithmic_bytes(wl, moved)
+    kern_ms = float(step_ms.mean())
+    achieved = a_step / (kern_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES.get(args.workload), "peak_source": peak_src,
+                "kernel": "fused_evict_kernel" if info["path"] == binding.KEYDIFF_PATH_FUSED else "staged chain (4 kernels)",
+                "algorithmic_bytes_per_launch": a_step, "moved_rows_per_unit": moved,
+                "kernel_ms": kern_ms, "kernel_ms_median": float(np.median(step_ms)),
+                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+
+    # ---- CPU baseline (the oracle as it stands) + a parity check of this very launch shape
+    cpu = None
+    if not args.no_cpu:
+        from oracle import compare, oracle
+        nk, nv = stream.next_block()
+        pre_k, pre_v = bits(k_cache), bits(v_cache)
+        cores = len(os.sched_getaffinity(0))
+        times, used = [], 1
+        for rep in range(3):
+            t0 = time.perf_counter()
+            out = oracle.evict_units_bf16(pre_k, pre_v, N, bits(nk), bits(nv), N, n_threads=cores)
+            times.append(time.perf_counter() - t0)
+            used = out["threads"]
+            if sum(times) > 12:
+                break
+        cpu = {"value": 1.0 / float(np.mean(times)), "unit": UNIT, "cores": used, "kind": "oracle",
+               "sample": f"{len(times)} evicting step(s), all {U} units, std::thread over units"}
+        kd.evict(k_cache, v_cache, nk, nv)
+        torch.cuda.synchronize()
+        sc = kd.scratch()
+        units = np.unique(np.linspace(0, U - 1, 16).astype(int))
+        rep = compare.check_step(pre_k, pre_v, N, bits(nk), bits(nv), N, bits(k_cache), bits(v_cache),
+                                 sc["scores"].cpu().numpy(), sc["kept_idx"].cpu().numpy(), units=units, n_threads=cores)
+        cpu["parity_units_checked"] = rep["units"]
+        cpu["max_score_err_over_tol"] = rep["max_score_err_over_tol"]
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": total_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 in, fp32 arithmetic", "data": "synthetic",
+            "config": {"workload": wl.name, "n_layers": wl.n_layers, "batch": wl.batch, "n_kv_heads": wl.n_kv_heads,
+                       "head_dim": d, "budget_N": N, "block_B": B, "units": U, "key_model": wl.key_model,
+                       "cache_bytes": 2 * U * N * d * 2, "l2_policy": "inputs larger than L2 (cache >> 126 MB)",
+                       "path": "fused" if info["path"] == binding.KEYDIFF_PATH_FUSED else "staged",
+                       "cluster_size": info["cluster_size"], "replicas": world},
+            "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": K * info["launches_per_step"],
+            "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line))
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on the host cores: each step scores/selects/gathers a bounded
+    sample of units of the same workload; the rate is scaled to whole steps."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle
+    wl = synth.WORKLOADS[args.workload]
+    sample_units = min(wl.units, 16)
+    small = synth.scaled(wl, n_layers=1, batch=1, n_kv_heads=sample_units)
+    k_cache, v_cache, stream = synth.prefilled_cache(small, "cpu")
+    kc, vc = bits(k_cache), bits(v_cache)
+    cores = len(os.sched_getaffinity(0))
+    K, W = args.steps, args.warmup
+    K = min(K, 20)
+    times, used = [], 1
+    for i in range(W + K):
+        nk, nv = stream.next_block()
+        t0 = time.perf_counter()
+        out = oracle.evict_units_bf16(kc, vc, small.budget, bits(nk), bits(nv), small.budget, n_threads=cores)
+        dt = time.perf_counter() - t0
+        kc, vc, used = out["k"], out["v"], out["threads"]
+        if i >= W:
+            times.append(dt)
+    per_step = float(np.mean(times)) * wl.units / sample_units
+    value = 1.0 / per_step
+    sample = f"{sample_units} of {wl.units} units per step, {K} steps, scaled to whole steps"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
+            "warmup": W, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "n_layers": wl.n_layers, "batch": wl.batch, "n_kv_heads": wl.n_kv_heads,
+                       "head_dim": wl.head_dim, "budget_N": wl.budget, "block_B": wl.block, "units": wl.units,
+                       "key_model": wl.key_model},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=189)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama31_8b_n8192", choices=list(synth.WORKLOADS))
+    ap.add_argument("--path", default="auto", choices=["auto", "staged", "fused"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
