@@ -55,7 +55,8 @@ enum {
     KEYDIFF_ERR_ALLOC = -3,       /* scratch allocation failed in keydiff_create */
     KEYDIFF_ERR_CUDA = -4,        /* a CUDA runtime call failed; see keydiff_last_cuda_error */
     KEYDIFF_ERR_STATE = -5,       /* call not valid in the ctx's current state */
-    KEYDIFF_ERR_TIMEOUT = -6      /* a bounded device-side wait expired (reported in the status word) */
+    KEYDIFF_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired (reported in the status word) */
+    KEYDIFF_ERR_TOO_LARGE = -7    /* keydiff_evict_static: the request does not fit the built-in scratch */
 };
 
 enum { KEYDIFF_BF16 = 0 };
@@ -164,6 +165,42 @@ KEYDIFF_API int keydiff_get_moved_rows(const keydiff_ctx* ctx, const unsigned lo
  * kernels launched per evicting step, cluster size (1 for the staged path). */
 KEYDIFF_API int keydiff_get_launch_info(const keydiff_ctx* ctx, int32_t* path, int32_t* launches_per_step,
                             int32_t* cluster_size);
+
+/*
+ * keydiff_evict_static -- the eviction step for callers that cannot allocate device memory.
+ * (The paper has no counterpart for this entry point; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside an inference server whose
+ * own memory pool has already claimed the GPU, in a plugin that is only ever handed tensors, or in
+ * a latency-critical loop where an allocation (which synchronises the device) is not acceptable.
+ * keydiff_create must allocate its scratch, so it is unusable there.  This call allocates nothing
+ * and frees nothing: its scratch is a 16 MiB array built into the library image (each GPU that
+ * loads the library carries those 16 MiB until the process exits).
+ *
+ * It computes exactly what keydiff_evict computes (staged kernels; same scores, same selection,
+ * same in-place compaction in token order), but keeps no context: the caller passes the current
+ * cache length `len` (0 <= len <= budget_N) and tracks the new one itself, min(budget_N, len +
+ * block_B).  k_cache/v_cache: device, in/out, [n_units][budget_N][128] bf16; new_k/new_v: device,
+ * read only, [n_units][block_B][128] bf16; all 16-byte aligned.  eps: 0 selects 1e-8.
+ * Asynchronous on `stream`.
+ *
+ * Limit: the step's scratch -- n_units * (8*(len+block_B) + 4*budget_N + 4) bytes plus the anchor
+ * partials, each part rounded up to 256 bytes -- must fit in 16 MiB (about 160 units at N=8192,
+ * B=128; about 2100 units at N=512, B=128) and len+block_B must not exceed 51200; otherwise the call
+ * returns KEYDIFF_ERR_TOO_LARGE and enqueues nothing.
+ *
+ * Set-up: the first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress) and sets one kernel attribute; the device must be current.  Make that
+ * first call before starting any stream capture.  Later calls do no set-up.
+ *
+ * Sharing: every call on a device uses the same array, and the array keeps whatever the previous
+ * call left in it (the call clears the one counter that has to start at zero).  Two calls whose
+ * GPU work can overlap -- different streams, or different host threads without ordering -- race
+ * on the scratch and corrupt each other; order them on one stream or with events.
+ */
+KEYDIFF_API int keydiff_evict_static(void* k_cache, void* v_cache, const void* new_k, const void* new_v,
+                                     int32_t len, int32_t budget_N, int32_t block_B, int32_t n_units,
+                                     int32_t head_dim, float eps, void* stream);
 
 /* Text of a status code; never NULL. */
 KEYDIFF_API const char* keydiff_strerror(int code);

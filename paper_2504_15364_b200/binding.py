@@ -17,13 +17,14 @@ LIB_PATH = _PKG / "libkeydiff.so"
 KEYDIFF_OK = 0
 KEYDIFF_ERR_INVALID_ARG, KEYDIFF_ERR_UNSUPPORTED, KEYDIFF_ERR_ALLOC = -1, -2, -3
 KEYDIFF_ERR_CUDA, KEYDIFF_ERR_STATE, KEYDIFF_ERR_TIMEOUT = -4, -5, -6
+KEYDIFF_ERR_TOO_LARGE = -7
 KEYDIFF_BF16 = 0
 KEYDIFF_PATH_AUTO, KEYDIFF_PATH_STAGED, KEYDIFF_PATH_FUSED = 0, 1, 2
 
 # every symbol include/keydiff.h declares
 EXPORTS = ["keydiff_create", "keydiff_evict", "keydiff_evict_host", "keydiff_destroy", "keydiff_reset",
            "keydiff_get_len", "keydiff_set_len", "keydiff_get_scratch", "keydiff_get_moved_rows",
-           "keydiff_get_launch_info",
+           "keydiff_get_launch_info", "keydiff_evict_static",
            "keydiff_strerror", "keydiff_last_cuda_error"]
 
 
@@ -64,6 +65,7 @@ def load_library() -> ctypes.CDLL:
     lib.keydiff_get_scratch.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.keydiff_get_moved_rows.argtypes = [vp, ctypes.POINTER(vp)]
     lib.keydiff_get_launch_info.argtypes = [vp, i32p, i32p, i32p]
+    lib.keydiff_evict_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, ctypes.c_float, vp]
     lib.keydiff_strerror.argtypes = [ctypes.c_int]
     lib.keydiff_strerror.restype = ctypes.c_char_p
     lib.keydiff_last_cuda_error.argtypes = []
@@ -189,3 +191,24 @@ class KeyDiff:
             self.close()
         except Exception:
             pass
+
+
+def evict_static(k_cache, v_cache, new_k, new_v, length: int, stream: torch.cuda.Stream | None = None,
+                 eps: float = 0.0) -> int:
+    """``keydiff_evict_static``: the eviction step without any device allocation, for callers that
+    may not call cudaMalloc (a server whose memory pool owns the GPU, a plugin that only receives
+    tensors).  Scratch is a 16 MiB array inside the library, shared by all calls on the device, so
+    calls must not overlap on the GPU.  Tensors are bf16 CUDA tensors [units, rows, 128]; ``length``
+    is the current cache length.  Returns the new length; raises KeyDiffError (TOO_LARGE) if the
+    step needs more than the built-in scratch."""
+    lib = load_library()
+    U, N, d = k_cache.shape
+    B = new_k.shape[1]
+    for t in (k_cache, v_cache, new_k, new_v):
+        if t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous():
+            raise KeyDiffError(KEYDIFF_ERR_INVALID_ARG, "need contiguous bf16 CUDA tensors")
+    assert v_cache.shape == k_cache.shape and new_k.shape == (U, B, d) and new_v.shape == (U, B, d)
+    st = (stream or torch.cuda.current_stream(k_cache.device)).cuda_stream
+    _check(lib.keydiff_evict_static(k_cache.data_ptr(), v_cache.data_ptr(), new_k.data_ptr(), new_v.data_ptr(),
+                                    length, N, B, U, d, eps, st))
+    return min(N, length + B)

@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstdlib>
+#include <mutex>
 #include <new>
 
 #include "common.cuh"
@@ -357,6 +358,7 @@ const char* keydiff_strerror(int code) {
         case KEYDIFF_ERR_CUDA: return "CUDA runtime error";
         case KEYDIFF_ERR_STATE: return "call not valid in the current state (is the ctx's device current?)";
         case KEYDIFF_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case KEYDIFF_ERR_TOO_LARGE: return "request needs more scratch than the built-in static scratch array holds";
         default: return "unknown keydiff status";
     }
 }
@@ -364,3 +366,109 @@ const char* keydiff_strerror(int code) {
 int keydiff_last_cuda_error(void) { return g_last_cuda_error; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free entry point.
+//
+// Some callers cannot allocate device memory at all: code running inside a serving process whose
+// memory pool already owns the whole GPU (any cudaMalloc would fail or fragment the pool), plugin
+// code that is only handed tensors, and set-ups where allocation is forbidden after start-up
+// because it synchronises the device.  keydiff_create needs cudaMalloc for its scratch, so such
+// callers get keydiff_evict_static instead: the same staged kernels, with their scratch carved
+// out of one array that is part of the library image.
+//
+// The array's name below is, in host code, only a handle for the runtime -- it is NOT a device
+// address, and a kernel handed it directly would read the wrong memory.  The device address is
+// looked up once per device with cudaGetSymbolAddress (with that device current) and cached.
+namespace {
+
+constexpr size_t kStaticScratchBytes = 16u << 20;   // 16 MiB, resident on every GPU that loads the library
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxStaticDevices = 64;
+unsigned char* g_static_scratch_addr[kMaxStaticDevices] = {};   // device address per device ordinal
+std::mutex g_static_mutex;
+
+// Resolve (once per device) the device address of the scratch array for the CURRENT device and
+// raise the select kernel's dynamic shared-memory limit there.
+int static_scratch_for_current_device(unsigned char** out) {
+    int dev = -1;
+    KD_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxStaticDevices) return KEYDIFF_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        int major = 0;
+        KD_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        if (major != 10) return KEYDIFF_ERR_UNSUPPORTED;
+        void* addr = nullptr;
+        KD_CUDA(cudaGetSymbolAddress(&addr, g_static_scratch));
+        KD_CUDA(cudaFuncSetAttribute(kd::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSelectSmem));
+        g_static_scratch_addr[dev] = static_cast<unsigned char*>(addr);
+    }
+    *out = g_static_scratch_addr[dev];
+    return KEYDIFF_OK;
+}
+
+inline size_t round256(size_t b) { return (b + 255) & ~static_cast<size_t>(255); }
+
+}  // namespace
+
+extern "C" int keydiff_evict_static(void* k_cache, void* v_cache, const void* new_k, const void* new_v,
+                                    int32_t len, int32_t budget_N, int32_t block_B, int32_t n_units,
+                                    int32_t head_dim, float eps, void* stream) {
+    using namespace kd;
+    if (!k_cache || !v_cache || !new_k || !new_v) return KEYDIFF_ERR_INVALID_ARG;
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(new_k) || !aligned16(new_v)) return KEYDIFF_ERR_INVALID_ARG;
+    if (k_cache == v_cache || k_cache == new_k || v_cache == new_v) return KEYDIFF_ERR_INVALID_ARG;
+    if (budget_N < 1 || block_B < 1 || n_units < 1 || len < 0 || len > budget_N || eps < 0.f) return KEYDIFF_ERR_INVALID_ARG;
+    if (head_dim != kHeadDim) return KEYDIFF_ERR_UNSUPPORTED;
+    if (n_units > 65535) return KEYDIFF_ERR_TOO_LARGE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint4* kc = static_cast<uint4*>(k_cache);
+    uint4* vc = static_cast<uint4*>(v_cache);
+    const uint4* nk = static_cast<const uint4*>(new_k);
+    const uint4* nv = static_cast<const uint4*>(new_v);
+    const long long n = static_cast<long long>(len) + block_B;
+    const int N = budget_N, U = n_units;
+    if (n <= N) {   // budget not exceeded: plain append, no scratch involved
+        const int threads = 256;
+        const dim3 grid((block_B * kRowVec + threads - 1) / threads, U, 2);
+        append_kernel<<<grid, threads, 0, st>>>(kc, vc, nk, nv, len, block_B, N);
+        KD_CUDA(cudaGetLastError());
+        return KEYDIFF_OK;
+    }
+    if (n * 4 > kMaxSelectSmem) return KEYDIFF_ERR_TOO_LARGE;
+    const int splits = static_cast<int>(std::max(1LL, std::min({(592LL + U - 1) / U, (n + 63) / 64, 64LL})));
+    // carve the static array: [moved counter][partials][norms][scores][kept_idx][first_evicted]
+    size_t off = 0;
+    auto take = [&off](size_t bytes) { const size_t o = off; off += round256(bytes); return o; };
+    const size_t o_moved = take(sizeof(unsigned long long));
+    const size_t o_partial = take(sizeof(float) * U * splits * kHeadDim);
+    const size_t o_norms = take(sizeof(float) * U * n);
+    const size_t o_scores = take(sizeof(float) * U * n);
+    const size_t o_kept = take(sizeof(int32_t) * static_cast<size_t>(U) * N);
+    const size_t o_first = take(sizeof(int32_t) * U);
+    if (off > kStaticScratchBytes) return KEYDIFF_ERR_TOO_LARGE;
+    unsigned char* base = nullptr;
+    const int src = static_scratch_for_current_device(&base);
+    if (src != KEYDIFF_OK) return src;
+    unsigned long long* moved = reinterpret_cast<unsigned long long*>(base + o_moved);
+    float* partial = reinterpret_cast<float*>(base + o_partial);
+    float* norms = reinterpret_cast<float*>(base + o_norms);
+    float* scores = reinterpret_cast<float*>(base + o_scores);
+    int32_t* kept = reinterpret_cast<int32_t*>(base + o_kept);
+    int32_t* first = reinterpret_cast<int32_t*>(base + o_first);
+    // the array still holds the previous call's contents; the counter accumulates, so it is the
+    // one part that must start from zero (everything else is fully overwritten before it is read)
+    KD_CUDA(cudaMemsetAsync(moved, 0, sizeof(unsigned long long), st));
+    const float e = eps > 0.f ? eps : kDefaultEps;
+    const int nn = static_cast<int>(n);
+    const int rows_per_split = (nn + splits - 1) / splits;
+    const dim3 grid(splits, U);
+    anchor_partial_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, len, block_B, N, e, rows_per_split, nn, partial, norms);
+    score_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, len, block_B, N, e, rows_per_split, nn, partial, norms, scores);
+    select_kernel<<<U, kSelectThreads, static_cast<size_t>(nn) * 4, st>>>(scores, nn, N, nn, len, kept, first, moved);
+    compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, len, block_B, N, kept, first);
+    KD_CUDA(cudaGetLastError());
+    return KEYDIFF_OK;
+}
