@@ -2,26 +2,30 @@
 // (one KV head of one layer of one sequence) from the anchor to the compacted K and V:
 //
 //   load K      every CTA pulls its contiguous slice of the unit's n key rows on chip exactly
-//               once: most rows into shared memory with TMA bulk copies (cp.async.bulk +
-//               mbarrier, all chunks in flight at once), the remainder into registers with
-//               128-bit loads.  Nothing is read from HBM twice.
-//   a1 anchor   per-row norm, sum of k/||k|| per CTA, partial sums combined across the cluster
-//               through distributed shared memory in a fixed order (App. B.1, expr. 1).
-//   a2 scores   e_i = -(mu.k_i)/max(||mu|| ||k_i||, eps) from the on-chip rows; the fp32 score goes
-//               to global scratch and its orderable key is pushed into every CTA's key table
-//               through DSMEM (App. B.1, expr. 2).
+//               once: most rows into shared memory with TMA bulk copies (cp.async.bulk, one
+//               mbarrier per 16-row tile), the remainder into registers with 128-bit loads.
+//               Nothing is read from HBM twice.
+//   a1 anchor   per-row norm, sum of k/||k|| per CTA; every CTA pushes its 128 partial sums into
+//               all peers' shared memory (DSMEM), one cluster barrier, then each CTA adds the C
+//               partials in rank order (App. B.1, expr. 1).
+//   a2 scores   e_i = -(mu.k_i)/max(||mu|| ||k_i||, eps) from the on-chip rows; the orderable key
+//               of e_i goes into this CTA's part of the key table, the part is then pushed to
+//               all peers with 128-bit DSMEM stores and one cluster barrier completes the table
+//               everywhere (App. B.1, expr. 2).  fp32 scores go to global scratch, coalesced.
 //   a3 select   every CTA finds the N-th largest key of the full table locally: a 2048-bin
-//               histogram over the (monotone) fixed-point image of e, then an exact rank among
-//               the few keys of the threshold bin; a 4x8-bit radix select is the fallback when
-//               that bin is crowded.  Ties keep the older token (Eq. efficient-keydiff, topk).
-//   a4 compact  an ordered scan gives every kept row its destination; K rows are written from
-//               chip to their new place, then the slice's V rows take the same trip (load all,
-//               cluster barrier, store all) -- in place, original token order (Eq. keydiff).
+//               histogram over a monotone fixed-point image of e, then an exact rank among the
+//               few keys of the threshold bin; a 4x8-bit radix select is the fallback when that
+//               bin is crowded.  Ties keep the older token (Eq. efficient-keydiff, topk).
+//   a4 compact  an ordered scan gives every kept row its destination; the rows then leave the
+//               chip tile by tile, and each shared-memory tile is refilled as soon as it has
+//               been written out: K stores hand their tile to the V load of the same rows, V
+//               stores hand it to the K load of the cluster's next unit.  The copy engine's
+//               loads therefore run under the stores (Eq. keydiff, in place, token order).
 //
-// In-place safety: every source row of the unit is on chip (in some CTA of the cluster)
-// before the first destination row is written -- for K by the barrier after the score pass, for
-// V by an explicit cluster barrier between its loads and its stores -- so no store can
-// overwrite a row that is still to be read.
+// In-place safety: every K row of the unit is on chip before the first cluster barrier, hence
+// before the first K store.  Every warp arrives at the third cluster barrier only after the V
+// rows it is responsible for have landed (bulk copies waited for, register loads consumed), and
+// no V store is issued before that barrier's wait: every V row that moves is then on chip.
 //
 // No multicast TMA is used anywhere; each CTA issues its own bulk loads.  Every mbarrier wait is
 // bounded: on expiry the kernel records KEYDIFF_ERR_TIMEOUT in the status word and carries on
@@ -36,35 +40,35 @@ namespace kd {
 constexpr int kFusedThreads = 512;
 constexpr int kFusedWarps = kFusedThreads / 32;
 constexpr int kGroups = kFusedThreads / kLanesPerRow;   // 64 row groups per CTA
-constexpr int kChunkRows = kGroups;                     // one bulk-load chunk = one row per group
-constexpr int kMaxChunks = 13;                          // <= 832 rows of a slice live in shared memory
-constexpr int kRegRows = 6;                             // + up to 6 rows per group (384 rows) in registers
-constexpr int kBins = 2048;                             // first-level histogram over e in [-1, 1]
+constexpr int kTileRows = 16;                           // one bulk copy = one tile of 16 rows (4 KB)
+constexpr int kMaxTiles = 52;                           // <= 832 rows of a slice live in shared memory
+constexpr int kTilesPerWarp = (kMaxTiles + kFusedWarps - 1) / kFusedWarps;
+constexpr int kMaxRegRows = 6;                          // + up to 6 rows per group (384 rows) in registers
+constexpr int kBins = 2048;                             // histogram over e in [-1, 1]
 constexpr int kCandCap = kFusedThreads;                 // exact-rank stage handles this many candidates
+constexpr int kMaxCluster = 16;
 constexpr int kSmemLimit = 232448;                      // opt-in shared memory per CTA on sm_100
 constexpr int kErrTimeout = -6;                         // KEYDIFF_ERR_TIMEOUT
 constexpr uint32_t kWaitSpins = 1u << 24;               // bound of every mbarrier wait
 
 struct FusedLayout {
-    int rows, keys, work, cand_key, cand_idx, norms, sel, partial, mu, mbar, misc, total;
+    int rows, keys, work, xchg, sel, mu, mbar, misc, total;
 };
 
-// Shared-memory carve-up for a slice with `smem_rows` resident rows and a key table of nkeys.
-__host__ __device__ inline FusedLayout fused_layout(int smem_rows, int nkeys) {
+// Shared-memory carve-up for a slice with `smem_rows` resident rows, a key table of nkeys
+// entries and a cluster of C CTAs.
+__host__ __device__ inline FusedLayout fused_layout(int smem_rows, int nkeys, int C) {
     FusedLayout L;
     int off = 0;
     auto take = [&off](int bytes) { const int o = off; off += (bytes + 127) & ~127; return o; };
     L.rows = take(smem_rows * kRowBytes);
     L.keys = take(nkeys * 4);
-    L.work = take(kBins * 4);   // histogram / warp-reduction scratch / destination table (never live together)
-    L.cand_key = take(kCandCap * 4);
-    L.cand_idx = take(kCandCap * 4);
-    L.norms = take(smem_rows * 4);
+    L.work = take(kBins * 4);   // warp-reduction scratch / histogram / destination table (never live together)
+    L.xchg = take(C * kHeadDim * 4 > 2 * kCandCap * 4 ? C * kHeadDim * 4 : 2 * kCandCap * 4);   // anchor partials [C][128] / candidates
     L.sel = take(static_cast<int>(sizeof(SelectSmem)));
-    L.partial = take(kHeadDim * 4);
     L.mu = take(kHeadDim * 4);
-    L.mbar = take(kMaxChunks * 8);
-    L.misc = take(64);
+    L.mbar = take(kMaxTiles * 8);
+    L.misc = take(128);
     L.total = off;
     return L;
 }
@@ -74,10 +78,11 @@ struct FusedParams {
     int len, B, N, U;
     float eps;
     int cluster;        // CTAs per cluster
-    int rows_per_cta;   // slice length = ceil(n / cluster)
-    int smem_rows;      // rows of a slice held in shared memory (multiple of kChunkRows)
-    int nkeys;          // key-table capacity (>= n)
+    int rows_per_cta;   // slice length = ceil(n / cluster) rounded up to a multiple of 4
+    int smem_rows;      // rows of a slice held in shared memory (multiple of kTileRows)
+    int nkeys;          // key-table capacity (>= cluster * rows_per_cta)
     int nmax;           // row stride of the score scratch
+    unsigned stagger_ns; // cluster c starts c * stagger_ns late (see the kernel)
     float* scores; int32_t* kept_idx; int32_t* first_evicted;
     unsigned long long* moved_rows; int32_t* status;
 };
@@ -85,18 +90,17 @@ struct FusedParams {
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_sync_all() { cluster_arrive(); cluster_wait(); }
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
     uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank)); return r;
 }
-__device__ __forceinline__ float ld_cluster_f32(uint32_t addr) {
-    float v; asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory"); return v;
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
-__device__ __forceinline__ void st_cluster_u32(uint32_t addr, uint32_t v) {
-    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, const uint4& v) {
+    asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -115,7 +119,9 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
+}
 
 // Bounded wait; returns false (and records the timeout) if the phase never completed.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status) {
@@ -125,279 +131,387 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t
     return false;
 }
 
-// fixed-point image of an orderable key: monotone non-decreasing in e, 2048 bins over [-1, 1]
+// inverse of order_key
+__device__ __forceinline__ float key_score(uint32_t key) {
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+// Histogram bin of an orderable key: e in [-1, 1] is shifted into the single binade [2, 4), where
+// the fp32 mantissa is a fixed-point image of the value; its top 11 bits are 2048 equal bins.  The
+// map is monotone non-decreasing in e (rounding and clamping are), which is all selection needs.
 __device__ __forceinline__ int key_bin(uint32_t key) {
-    const uint32_t u = (key & 0x80000000u) ? (key & 0x7fffffffu) : ~key;   // inverse of order_key
-    const int q = __float2int_rd((__uint_as_float(u) + 1.0f) * 1024.0f);
-    return min(max(q, 0), kBins - 1);
+    const float f = fmaxf(fminf(key_score(key) + 3.0f, 3.9999998f), 2.0f);
+    return static_cast<int>((__float_as_uint(f) >> 12) & (kBins - 1));
 }
 
-// Thread 0: start the bulk loads of this CTA's resident rows [0, rs) of a slice starting at unit
-// row seg_a, one mbarrier per chunk of 64 rows; chunks that end at or before skip_local are left
-// out.  Rows below `len` come from the cache tensor, the rest from the block tensor.
-__device__ __forceinline__ void issue_slice_loads(const uint4* cache, const uint4* block, int u, int len, int B, int N,
-                                                  int seg_a, int rs, int skip_local, uint32_t rows_sa, uint32_t mbar_sa) {
-    for (int j = 0; j * kChunkRows < rs; ++j) {
-        const int lo = j * kChunkRows, hi = min(rs, lo + kChunkRows);
-        if (hi <= skip_local) continue;
-        const int g0 = seg_a + lo;                               // first unit row of the chunk
-        const int from_cache = min(max(len - g0, 0), hi - lo);
-        const int from_block = (hi - lo) - from_cache;
-        const uint32_t bar = mbar_sa + 8 * j, dst = rows_sa + lo * kRowBytes;
-        mbar_expect_tx(bar, (hi - lo) * kRowBytes);
-        if (from_cache > 0)
-            bulk_load(dst, cache + (static_cast<size_t>(u) * N + g0) * kRowVec, from_cache * kRowBytes, bar);
-        if (from_block > 0)
-            bulk_load(dst + from_cache * kRowBytes,
-                      block + (static_cast<size_t>(u) * B + (g0 + from_cache - len)) * kRowVec, from_block * kRowBytes, bar);
+// Geometry of one CTA's slice of a unit (identical for every unit of a step).
+struct Slice {
+    int seg_a, seg;     // first unit row, number of rows
+    int rs;             // rows resident in shared memory (the first rs of the slice)
+    int ntiles;         // ceil(rs / kTileRows)
+};
+
+// One thread: start the bulk load of tile `tile` (local rows [16*tile, min(rs, 16*tile+16))) of unit
+// u's slice on that tile's mbarrier.  Rows below `len` come from the cache tensor, the rest from
+// the block tensor.
+__device__ __forceinline__ void issue_tile(const uint4* cache, const uint4* block, int u, int len, int B, int N,
+                                           const Slice& s, int tile, uint32_t rows_sa, uint32_t mbar_sa) {
+    const int lo = tile * kTileRows, hi = min(s.rs, lo + kTileRows);
+    const int g0 = s.seg_a + lo;                               // first unit row of the tile
+    const int from_cache = min(max(len - g0, 0), hi - lo);
+    const int from_block = (hi - lo) - from_cache;
+    const uint32_t bar = mbar_sa + 8 * tile, dst = rows_sa + lo * kRowBytes;
+    mbar_expect_tx(bar, (hi - lo) * kRowBytes);
+    if (from_cache > 0)
+        bulk_load(dst, cache + (static_cast<size_t>(u) * N + g0) * kRowVec, from_cache * kRowBytes, bar);
+    if (from_block > 0)
+        bulk_load(dst + from_cache * kRowBytes,
+                  block + (static_cast<size_t>(u) * B + (g0 + from_cache - len)) * kRowVec, from_block * kRowBytes, bar);
+}
+
+// ---------------------------------------------------------------- row arithmetic (packed fp32 pairs)
+// A lane's two 128-bit words of a row as 8 fp32 pairs; pair p holds channels lane_channel(t, 2p) and
+// lane_channel(t, 2p + 1).
+__device__ __forceinline__ void unpack_pairs(const uint4& a, const uint4& b, float2 (&x)[8]) {
+    x[0] = make_float2(bf16_lo(a.x), bf16_hi(a.x)); x[1] = make_float2(bf16_lo(a.y), bf16_hi(a.y));
+    x[2] = make_float2(bf16_lo(a.z), bf16_hi(a.z)); x[3] = make_float2(bf16_lo(a.w), bf16_hi(a.w));
+    x[4] = make_float2(bf16_lo(b.x), bf16_hi(b.x)); x[5] = make_float2(bf16_lo(b.y), bf16_hi(b.y));
+    x[6] = make_float2(bf16_lo(b.z), bf16_hi(b.z)); x[7] = make_float2(bf16_lo(b.w), bf16_hi(b.w));
+}
+__device__ __forceinline__ float approx_rsqrt(float v) { float r; asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v)); return r; }
+__device__ __forceinline__ float approx_sqrt(float v) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v)); return r; }
+__device__ __forceinline__ float approx_rcp(float v) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v)); return r; }
+
+// ||k||^2 over the row group (two FMA chains per lane, then the 8-lane butterfly)
+__device__ __forceinline__ float pairs_sumsq(const float2 (&x)[8]) {
+    float2 s0 = make_float2(0.f, 0.f), s1 = s0;
+#pragma unroll
+    for (int p = 0; p < 4; ++p) { s0 = __ffma2_rn(x[p], x[p], s0); s1 = __ffma2_rn(x[4 + p], x[4 + p], s1); }
+    return group_sum((s0.x + s0.y) + (s1.x + s1.y));
+}
+__device__ __forceinline__ float pairs_dot(const float2 (&x)[8], const float2 (&w)[8]) {
+    float2 s0 = make_float2(0.f, 0.f), s1 = s0;
+#pragma unroll
+    for (int p = 0; p < 4; ++p) { s0 = __ffma2_rn(x[p], w[p], s0); s1 = __ffma2_rn(x[4 + p], w[4 + p], s1); }
+    return group_sum((s0.x + s0.y) + (s1.x + s1.y));
+}
+// Step a1 for one row: returns ||k||; adds k / max(||k||, eps) into acc when the row is valid.
+// 1/max(r, eps) = min(1/r, 1/eps); the reciprocal square root and the square root are the
+// hardware approximations (relative error about 2^-22, far inside the score tolerance).
+__device__ __forceinline__ float row_a1(const uint4& a, const uint4& b, bool valid, float inv_eps, float2 (&acc)[8]) {
+    float2 x[8];
+    unpack_pairs(a, b, x);
+    const float ss = pairs_sumsq(x);
+    const float inv = valid ? fminf(approx_rsqrt(ss), inv_eps) : 0.f;
+    const float2 inv2 = make_float2(inv, inv);
+#pragma unroll
+    for (int p = 0; p < 8; ++p) acc[p] = __ffma2_rn(x[p], inv2, acc[p]);
+    return approx_sqrt(ss);
+}
+// Step a2 for one row: orderable key of e = -(mu.k)/max(||mu|| ||k||, eps), -0 mapped to +0.
+__device__ __forceinline__ uint32_t row_a2(const uint4& a, const uint4& b, const float2 (&w)[8], float m, float r, float eps) {
+    float2 x[8];
+    unpack_pairs(a, b, x);
+    const float dot = pairs_dot(x, w);
+    const float e = -(dot * approx_rcp(fmaxf(m * r, eps)));
+    return order_key(e == 0.f ? 0.f : e);
+}
+
+// Exact top-N over the whole key table by one CTA (every CTA of the cluster runs it on its own
+// copy and gets the same answer): 2048-bin histogram, exact rank inside the threshold bin, radix
+// select when that bin is crowded; then an ordered scan gives every kept row of this CTA's slice
+// its destination (-1 = evicted) and misc[1] the index of the first evicted token.
+__device__ __noinline__ void full_select_plan(const uint32_t* keys, int n, int N, int seg_a, int seg_b, int* hist,
+                                              uint32_t* cand_key, int* cand_idx, int* dst_of, SelectSmem& sel, int* misc) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;
+    if (tid == 0) { misc[0] = 0; misc[1] = n; }
+    __syncthreads();
+    // thread t owns the tokens [i0, i1): an odd stride keeps the shared-memory reads conflict-free
+    const int per = ((n + kFusedThreads - 1) / kFusedThreads) | 1;
+    const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
+    for (int i = i0; i < i1; ++i) atomicAdd(&hist[key_bin(keys[i])], 1);
+    __syncthreads();
+    {
+        // thread t owns bins 2047-4t .. 2044-4t (descending); find the bin holding rank N
+        int c4[4], tot = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { c4[q] = hist[kBins - 1 - 4 * tid - q]; tot += c4[q]; }
+        int incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) sel.warp_gt[warp] = incl;
+        __syncthreads();
+        int before = 0;
+        for (int w = 0; w < warp; ++w) before += sel.warp_gt[w];
+        incl += before;
+        const int excl = incl - tot;
+        if (excl < N && N <= incl) {
+            int above = excl;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (above < N && N <= above + c4[q]) { sel.bcast[0] = kBins - 1 - 4 * tid - q; sel.bcast[1] = above; }
+                above += c4[q];
+            }
+        }
+        __syncthreads();
     }
+    const int bstar = sel.bcast[0];
+    const int need = N - sel.bcast[1];       // tokens of the threshold bin that are kept, >= 1
+    for (int j = 0; j < per; ++j) {          // same trip count in every lane: the ballot is warp-wide
+        const int i = i0 + j;
+        const uint32_t k = i < i1 ? keys[i] : 0u;
+        const bool inbin = i < i1 && key_bin(k) == bstar;
+        const unsigned peers = __ballot_sync(0xffffffffu, inbin);
+        if (peers != 0) {                    // one shared-memory atomic per warp, not per candidate
+            const int leader = __ffs(peers) - 1;
+            int base = 0;
+            if (lane == leader) base = atomicAdd(&misc[0], __popc(peers));
+            base = __shfl_sync(0xffffffffu, base, leader);
+            const int slot = base + __popc(peers & ((1u << lane) - 1u));
+            if (inbin && slot < kCandCap) { cand_key[slot] = k; cand_idx[slot] = i; }
+        }
+    }
+    __syncthreads();
+    Threshold th;
+    const int ncand = misc[0];
+    if (ncand <= kCandCap) {
+        // exact rank among the candidates under (key desc, index asc): one candidate per warp at a
+        // time, its comparisons spread over the lanes
+        for (int c = warp; c < ncand; c += kFusedWarps) {
+            const uint32_t mk = cand_key[c];
+            const int mi = cand_idx[c];
+            int rank = 0, eq_older = 0;
+            for (int q = lane; q < ncand; q += 32) {
+                const uint32_t ok = cand_key[q];
+                const int oi = cand_idx[q];
+                rank += (ok > mk) || (ok == mk && oi < mi);
+                eq_older += (ok == mk && oi <= mi);
+            }
+            rank = __reduce_add_sync(0xffffffffu, rank);
+            eq_older = __reduce_add_sync(0xffffffffu, eq_older);
+            if (lane == 0 && rank == need - 1) { misc[3] = static_cast<int>(mk); misc[2] = eq_older; }
+        }
+        __syncthreads();
+        th.key = static_cast<uint32_t>(misc[3]);
+        th.need_eq = misc[2];
+    } else {
+        th = block_radix_select<kFusedThreads>(keys, n, N, sel);
+    }
+    int gt = 0, eq = 0;
+    for (int i = i0; i < i1; ++i) { const uint32_t k = keys[i]; gt += k > th.key; eq += k == th.key; }
+    int pre_gt, pre_eq, tot_gt, tot_eq;
+    block_exclusive_scan2<kFusedThreads>(gt, eq, sel, pre_gt, pre_eq, tot_gt, tot_eq);   // syncs: hist is dead
+    int local_first = n;
+    for (int i = i0; i < i1; ++i) {
+        const uint32_t k = keys[i];
+        const bool is_eq = k == th.key;
+        const bool keep = k > th.key || (is_eq && pre_eq < th.need_eq);
+        if (i >= seg_a && i < seg_b) dst_of[i - seg_a] = keep ? pre_gt + min(pre_eq, th.need_eq) : -1;
+        if (!keep) local_first = min(local_first, i);
+        pre_gt += k > th.key;
+        pre_eq += is_eq;
+    }
+    if (local_first < n) atomicMin(&misc[1], local_first);
+    __syncthreads();
 }
 
+// kRegRows = rows per row group that live in registers (the host picks the smallest instance that
+// holds a slice together with the shared-memory rows).
+template <int kRegRows>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const FusedParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    const FusedLayout L = fused_layout(p.smem_rows, p.nkeys);
+    const int C = p.cluster;
+    const FusedLayout L = fused_layout(p.smem_rows, p.nkeys, C);
     uint4* rows = reinterpret_cast<uint4*>(smem + L.rows);
     uint32_t* keys = reinterpret_cast<uint32_t*>(smem + L.keys);
     int* hist = reinterpret_cast<int*>(smem + L.work);
     float* red = reinterpret_cast<float*>(smem + L.work);
     int* dst_of = reinterpret_cast<int*>(smem + L.work);
-    uint32_t* cand_key = reinterpret_cast<uint32_t*>(smem + L.cand_key);
-    int* cand_idx = reinterpret_cast<int*>(smem + L.cand_idx);
-    float* norms = reinterpret_cast<float*>(smem + L.norms);
+    float* partials = reinterpret_cast<float*>(smem + L.xchg);          // [C][128], filled by the peers
+    uint32_t* cand_key = reinterpret_cast<uint32_t*>(smem + L.xchg);
+    int* cand_idx = reinterpret_cast<int*>(smem + L.xchg) + kCandCap;
     SelectSmem& sel = *reinterpret_cast<SelectSmem*>(smem + L.sel);
-    float* partial = reinterpret_cast<float*>(smem + L.partial);
     float* mu_sh = reinterpret_cast<float*>(smem + L.mu);
-    int* misc = reinterpret_cast<int*>(smem + L.misc);   // 0 ncand, 1 first_evicted, 2 need_eq, 3 T, 4 winner idx, 5 m (float)
+    int* misc = reinterpret_cast<int*>(smem + L.misc);   // 0 ncand, 1 first_evicted, 2 need_eq, 3 threshold key
     const uint32_t rows_sa = smem_addr(rows), mbar_sa = smem_addr(smem + L.mbar);
-    const uint32_t keys_sa = smem_addr(keys), partial_sa = smem_addr(partial);
+    const uint32_t keys_sa = smem_addr(keys), partials_sa = smem_addr(partials);
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = tid >> 3, t = tid & 7;
-    const int C = p.cluster;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = tid >> 3, t = tid & 7, sub = lane >> 3;
     const int crank = static_cast<int>(cluster_ctarank());
     const int cluster_id = blockIdx.x / C, nclusters = gridDim.x / C;
     const int len = p.len, B = p.B, N = p.N, n = len + B;
-    const int seg_a = min(n, crank * p.rows_per_cta), seg_b = min(n, seg_a + p.rows_per_cta), seg = seg_b - seg_a;
-    const int rs = min(seg, p.smem_rows);            // slice rows resident in shared memory
-    const int nchunks = (rs + kChunkRows - 1) / kChunkRows;
+    const float inv_eps = 1.0f / p.eps;
+    Slice sl;
+    sl.seg_a = min(n, crank * p.rows_per_cta);
+    sl.seg = min(n, sl.seg_a + p.rows_per_cta) - sl.seg_a;
+    sl.rs = min(sl.seg, p.smem_rows);
+    sl.ntiles = (sl.rs + kTileRows - 1) / kTileRows;
+    const int seg_a = sl.seg_a, seg = sl.seg, seg_b = seg_a + seg, rs = sl.rs, ntiles = sl.ntiles;
+    // Shared-memory rows are handled tile by tile (16 rows); warp w owns tiles w, w+16, w+32, ... in
+    // every phase, so a tile is loaded, read, written out and refilled by one warp: the hand-over of
+    // a tile from its readers to the copy engine needs a __syncwarp, never a CTA-wide barrier.
 
     if (tid == 0) {
-        for (int j = 0; j < kMaxChunks; ++j) mbar_init(mbar_sa + 8 * j, 1);
+        for (int j = 0; j < kMaxTiles; ++j) mbar_init(mbar_sa + 8 * j, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    uint32_t parity = 0;   // bit j: phase parity the next wait on chunk j's mbarrier expects
+    uint32_t parity = 0;   // bit s: phase parity the next wait on this warp's s-th tile expects
 
-    for (int u = cluster_id; u < p.U; u += nclusters) {
-        // ------------------------------------------------------------ load K (once)
-        if (tid == 0) {
-            fence_proxy_async();
-            issue_slice_loads(p.k_cache, p.new_k, u, len, B, N, seg_a, rs, -1, rows_sa, mbar_sa);
-        }
-        uint4 ra[kRegRows], rb[kRegRows];   // register-resident rows: local row rs + 64k + g
-        float rn[kRegRows];
+    // All clusters start together and do identical work per unit, so left alone they stay in lock
+    // step: every SM loads at the same moment, then every SM computes while HBM idles.  Starting
+    // cluster c a fraction of a unit's duration late spreads the memory phases over time.  Clusters
+    // with the lower ids are also the ones that may own one unit more, so the delay mostly fills
+    // slack that the uneven unit count leaves anyway.  The wait is bounded.
+    if (p.stagger_ns != 0 && cluster_id != 0) {
+        const unsigned long long t0 = global_timer_ns();
+        const unsigned long long wait_ns = static_cast<unsigned long long>(p.stagger_ns) * static_cast<unsigned>(cluster_id);
+        for (int spin = 0; spin < (1 << 16) && global_timer_ns() - t0 < wait_ns; ++spin) __nanosleep(100);
+    }
+
+    constexpr int kRegSlots = kRegRows > 0 ? kRegRows : 1;   // no zero-sized arrays in device code
+    uint4 ra[kRegSlots], rb[kRegSlots];   // register-resident rows: local row rs + 64k + g
+    float rn[kRegSlots];
+    // K of the cluster's first unit: tiles by the copy engine, the rest by plain loads
+    if (cluster_id < p.U) {
+        if (lane < kTilesPerWarp && warp + kFusedWarps * lane < ntiles)
+            issue_tile(p.k_cache, p.new_k, cluster_id, len, B, N, sl, warp + kFusedWarps * lane, rows_sa, mbar_sa);
 #pragma unroll
         for (int k = 0; k < kRegRows; ++k) {
             const int lr = rs + k * kGroups + g;
             ra[k] = make_uint4(0, 0, 0, 0); rb[k] = ra[k];
             if (lr < seg) {
-                const uint4* row = concat_row(p.k_cache, p.new_k, u, seg_a + lr, len, B, N);
+                const uint4* row = concat_row(p.k_cache, p.new_k, cluster_id, seg_a + lr, len, B, N);
                 ra[k] = row[t]; rb[k] = row[t + 8];
             }
         }
+    }
+
+    for (int u = cluster_id; u < p.U; u += nclusters) {
+        const int un = u + nclusters;   // the unit this cluster serves next
         // ------------------------------------------------------------ a1: norms and anchor partial
-        float acc[16];
+        float2 acc[8];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) acc[j] = 0.f;
-        for (int j = 0; j < nchunks; ++j) {
-            mbar_wait(mbar_sa + 8 * j, (parity >> j) & 1u, p.status);
-            const int lr = j * kChunkRows + g;
-            const bool valid = lr < rs;
-            uint4 a = make_uint4(0, 0, 0, 0), b = a;
-            if (valid) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
-            float x[16];
-            unpack_row(a, b, x);
-            const float r = sqrtf(row_sumsq(x));
-            const float inv = 1.0f / fmaxf(r, p.eps);
-            if (valid) {
+        for (int q = 0; q < 8; ++q) acc[q] = make_float2(0.f, 0.f);
+#pragma unroll 1
+        for (int s = 0; s < kTilesPerWarp; ++s) {
+            const int tile = warp + kFusedWarps * s;
+            if (tile >= ntiles) break;
+            mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
+            parity ^= 1u << s;
+#pragma unroll 1
+            for (int half = 0; half < 2; ++half) {
+                uint4 a[2], b[2];
 #pragma unroll
-                for (int q = 0; q < 16; ++q) acc[q] = fmaf(x[q], inv, acc[q]);
-                if (t == 0) norms[lr] = r;
+                for (int it = 0; it < 2; ++it) {
+                    const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
+                    a[it] = make_uint4(0, 0, 0, 0); b[it] = a[it];
+                    if (lr < rs) { a[it] = rows[lr * kRowVec + t]; b[it] = rows[lr * kRowVec + t + 8]; }
+                }
+#pragma unroll
+                for (int it = 0; it < 2; ++it) {
+                    const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
+                    const float r = row_a1(a[it], b[it], lr < rs, inv_eps, acc);
+                    if (lr < rs && t == 0) keys[seg_a + lr] = __float_as_uint(r);   // parked in the row's key slot until a2
+                }
             }
         }
-        parity ^= (1u << nchunks) - 1u;
 #pragma unroll
-        for (int k = 0; k < kRegRows; ++k) {
-            float x[16];
-            unpack_row(ra[k], rb[k], x);
-            const float r = sqrtf(row_sumsq(x));
-            const float inv = 1.0f / fmaxf(r, p.eps);
-            rn[k] = r;
-            if (rs + k * kGroups + g < seg) {
-#pragma unroll
-                for (int q = 0; q < 16; ++q) acc[q] = fmaf(x[q], inv, acc[q]);
-            }
-        }
+        for (int k = 0; k < kRegRows; ++k) rn[k] = row_a1(ra[k], rb[k], rs + k * kGroups + g < seg, inv_eps, acc);
         // CTA reduction: 4 groups of a warp by shuffle, 16 warps through shared memory, fixed order
 #pragma unroll
-        for (int q = 0; q < 16; ++q) {
-            float v = acc[q];
-            v += __shfl_xor_sync(0xffffffffu, v, 8);
-            v += __shfl_xor_sync(0xffffffffu, v, 16);
+        for (int q = 0; q < 8; ++q) {
+            float2 v = acc[q];
+            v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
+            v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
             acc[q] = v;
         }
         if (lane < 8) {
 #pragma unroll
-            for (int q = 0; q < 16; ++q) red[warp * kHeadDim + lane_channel(t, q)] = acc[q];
+            for (int q = 0; q < 8; ++q)
+                *reinterpret_cast<float2*>(&red[warp * kHeadDim + lane_channel(t, 2 * q)]) = acc[q];
         }
         __syncthreads();
         if (tid < kHeadDim) {
             float s = 0.f;
+#pragma unroll
             for (int w = 0; w < kFusedWarps; ++w) s += red[w * kHeadDim + tid];
-            partial[tid] = s;
+            const uint32_t slot = partials_sa + 4 * (crank * kHeadDim + tid);
+            for (int c = 0; c < C; ++c) st_cluster_f32(map_to_cta(slot, c), s);   // this CTA's row of every peer's table
         }
-        cluster_sync_all();   // (1) every CTA's partial is written; all K rows of the unit are on chip
+        cluster_sync_all();   // (1) all partials delivered; every K row of the unit is on chip
         if (tid < kHeadDim) {
             float s = 0.f;
-            for (int c = 0; c < C; ++c) s += ld_cluster_f32(map_to_cta(partial_sa + 4 * tid, c));   // fixed order
+            for (int c = 0; c < C; ++c) s += partials[c * kHeadDim + tid];   // rank order: same bits in every CTA
             mu_sh[tid] = s / static_cast<float>(n);
         }
         __syncthreads();
-        if (warp == 0) {
-            float v = 0.f;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) { const float w = mu_sh[lane * 4 + q]; v = fmaf(w, w, v); }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (lane == 0) reinterpret_cast<float*>(misc)[5] = sqrtf(v);
-        }
-        __syncthreads();
-        // ------------------------------------------------------------ a2: scores, keys pushed to every CTA
+        // ------------------------------------------------------------ a2: keys of this slice into the table
         {
-            float w[16];
+            float2 w[8];
 #pragma unroll
-            for (int q = 0; q < 16; ++q) w[q] = mu_sh[lane_channel(t, q)];
-            const float m = reinterpret_cast<float*>(misc)[5];
-            for (int j = 0; j < nchunks; ++j) {
-                const int lr = j * kChunkRows + g;
-                const bool valid = lr < rs;
-                uint4 a = make_uint4(0, 0, 0, 0), b = a;
-                if (valid) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
-                float x[16];
-                unpack_row(a, b, x);
-                const float dot = row_dot(x, w);
-                if (valid) {
-                    const float e = eviction_score(dot, m, norms[lr], p.eps);
-                    const int i = seg_a + lr;
-                    if (t == 0) p.scores[static_cast<size_t>(u) * p.nmax + i] = e;
-                    const uint32_t key = order_key(e);
-                    for (int c = t; c < C; c += kLanesPerRow) st_cluster_u32(map_to_cta(keys_sa + 4 * i, c), key);
+            for (int q = 0; q < 8; ++q) w[q] = *reinterpret_cast<const float2*>(&mu_sh[lane_channel(t, 2 * q)]);
+            float m;   // ||mu||, computed by every warp in the same order
+            {
+                const float4 c4 = reinterpret_cast<const float4*>(mu_sh)[lane];
+                float v = fmaf(c4.w, c4.w, fmaf(c4.z, c4.z, fmaf(c4.y, c4.y, c4.x * c4.x)));
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                m = sqrtf(v);
+            }
+#pragma unroll 1
+            for (int s = 0; s < kTilesPerWarp; ++s) {
+                const int tile = warp + kFusedWarps * s;
+                if (tile >= ntiles) break;
+#pragma unroll 1
+                for (int half = 0; half < 2; ++half) {
+                    uint4 a[2], b[2];
+                    float r[2];
+#pragma unroll
+                    for (int it = 0; it < 2; ++it) {
+                        const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
+                        a[it] = make_uint4(0, 0, 0, 0); b[it] = a[it]; r[it] = 0.f;
+                        if (lr < rs) { a[it] = rows[lr * kRowVec + t]; b[it] = rows[lr * kRowVec + t + 8]; r[it] = __uint_as_float(keys[seg_a + lr]); }
+                    }
+#pragma unroll
+                    for (int it = 0; it < 2; ++it) {
+                        const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
+                        const uint32_t key = row_a2(a[it], b[it], w, m, r[it], p.eps);
+                        if (lr < rs && t == 0) keys[seg_a + lr] = key;
+                    }
                 }
             }
 #pragma unroll
             for (int k = 0; k < kRegRows; ++k) {
-                float x[16];
-                unpack_row(ra[k], rb[k], x);
-                const float dot = row_dot(x, w);
+                const uint32_t key = row_a2(ra[k], rb[k], w, m, rn[k], p.eps);
                 const int lr = rs + k * kGroups + g;
-                if (lr < seg) {
-                    const float e = eviction_score(dot, m, rn[k], p.eps);
-                    const int i = seg_a + lr;
-                    if (t == 0) p.scores[static_cast<size_t>(u) * p.nmax + i] = e;
-                    const uint32_t key = order_key(e);
-                    for (int c = t; c < C; c += kLanesPerRow) st_cluster_u32(map_to_cta(keys_sa + 4 * i, c), key);
-                }
+                if (lr < seg && t == 0) keys[seg_a + lr] = key;
             }
         }
-        cluster_sync_all();   // (2) the key table of every CTA holds all n keys
-        // ------------------------------------------------------------ a3: N-th largest key
-        for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;
-        if (tid == 0) { misc[0] = 0; misc[1] = n; misc[2] = 0; }
-        __syncthreads();
-        for (int i = tid; i < n; i += kFusedThreads) atomicAdd(&hist[key_bin(keys[i])], 1);
         __syncthreads();
         {
-            // thread t owns bins 2047-4t .. 2044-4t (descending); find the bin holding rank N
-            int c4[4], tot = 0;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) { c4[q] = hist[kBins - 1 - 4 * tid - q]; tot += c4[q]; }
-            int incl = tot;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            if (lane == 31) sel.warp_gt[warp] = incl;
-            __syncthreads();
-            int before = 0;
-            for (int w = 0; w < warp; ++w) before += sel.warp_gt[w];
-            incl += before;
-            const int excl = incl - tot;
-            if (excl < N && N <= incl) {
-                int above = excl;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    if (above < N && N <= above + c4[q]) { sel.bcast[0] = kBins - 1 - 4 * tid - q; sel.bcast[1] = above; }
-                    above += c4[q];
-                }
-            }
-            __syncthreads();
-        }
-        const int bstar = sel.bcast[0];
-        const int need = N - sel.bcast[1];       // tokens of the threshold bin that are kept, >= 1
-        for (int i = tid; i < n; i += kFusedThreads) {
-            const uint32_t k = keys[i];
-            if (key_bin(k) == bstar) {
-                const int slot = atomicAdd(&misc[0], 1);
-                if (slot < kCandCap) { cand_key[slot] = k; cand_idx[slot] = i; }
+            // this slice's keys -> every peer's table (128-bit DSMEM stores)
+            const uint4* mine = reinterpret_cast<const uint4*>(keys + seg_a);
+            for (int c = 1; c < C; ++c) {
+                const int peer = crank + c < C ? crank + c : crank + c - C;
+                const uint32_t base = map_to_cta(keys_sa + 4 * seg_a, peer);
+                for (int o = tid; 4 * o < seg; o += kFusedThreads) st_cluster_v4(base + 16 * o, mine[o]);
             }
         }
-        __syncthreads();
-        Threshold th;
-        const int ncand = misc[0];
-        if (ncand <= kCandCap) {
-            // exact rank among the candidates under (key desc, index asc)
-            if (tid < ncand) {
-                const uint32_t mk = cand_key[tid];
-                const int mi = cand_idx[tid];
-                int rank = 0;
-                for (int q = 0; q < ncand; ++q) {
-                    const uint32_t ok = cand_key[q];
-                    rank += (ok > mk) || (ok == mk && cand_idx[q] < mi);
-                }
-                if (rank == need - 1) { misc[3] = static_cast<int>(mk); misc[4] = mi; }
-            }
-            __syncthreads();
-            if (tid < ncand && cand_key[tid] == static_cast<uint32_t>(misc[3]) && cand_idx[tid] <= misc[4])
-                atomicAdd(&misc[2], 1);
-            __syncthreads();
-            th.key = static_cast<uint32_t>(misc[3]);
-            th.need_eq = misc[2];
-        } else {
-            th = block_radix_select<kFusedThreads>(keys, n, N, sel);
-        }
-        // ------------------------------------------------------------ plan: destination of every kept row
+        cluster_arrive();
         {
-            const int per = (n + kFusedThreads - 1) / kFusedThreads;
-            const int i0 = min(n, tid * per), i1 = min(n, i0 + per);
-            int gt = 0, eq = 0;
-            for (int i = i0; i < i1; ++i) { const uint32_t k = keys[i]; gt += k > th.key; eq += k == th.key; }
-            int pre_gt, pre_eq, tot_gt, tot_eq;
-            block_exclusive_scan2<kFusedThreads>(gt, eq, sel, pre_gt, pre_eq, tot_gt, tot_eq);
-            int local_first = n;
-            for (int i = i0; i < i1; ++i) {
-                const uint32_t k = keys[i];
-                const bool is_eq = k == th.key;
-                const bool keep = k > th.key || (is_eq && pre_eq < th.need_eq);
-                if (i >= seg_a && i < seg_b) dst_of[i - seg_a] = keep ? pre_gt + min(pre_eq, th.need_eq) : -1;
-                if (!keep) local_first = min(local_first, i);
-                pre_gt += k > th.key;
-                pre_eq += is_eq;
-            }
-            if (local_first < n) atomicMin(&misc[1], local_first);
-            __syncthreads();
+            float* sc = p.scores + static_cast<size_t>(u) * p.nmax + seg_a;   // fp32 scores to global scratch, coalesced
+            for (int lr = tid; lr < seg; lr += kFusedThreads) sc[lr] = key_score(keys[seg_a + lr]);
         }
+        cluster_wait();       // (2) the key table of every CTA holds all n keys
+        // ------------------------------------------------------------ a3 + plan: who is evicted, where every kept row goes
+        full_select_plan(keys, n, N, seg_a, seg_b, hist, cand_key, cand_idx, dst_of, sel, misc);
         const int first_evicted = misc[1];
         const int first_moved = min(first_evicted, len);   // block rows always move into the cache
+        const int skip_local = first_moved - seg_a;        // local rows below this keep their place
         if (crank == 0 && tid == 0) {
             p.first_evicted[u] = first_evicted;
             atomicAdd(p.moved_rows, static_cast<unsigned long long>(N - first_moved));
@@ -406,49 +520,60 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             const int d = dst_of[lr];
             if (d >= 0) p.kept_idx[static_cast<size_t>(u) * N + d] = seg_a + lr;
         }
-        // ------------------------------------------------------------ a4: K rows to their new place
+        // ------------------------------------------------------------ a4: K rows out, V rows in behind them
         {
             uint4* out = p.k_cache + static_cast<size_t>(u) * N * kRowVec;
-            for (int q = tid; q < rs * kRowVec; q += kFusedThreads) {
-                const int lr = q >> 4, d = dst_of[lr];
-                if (d >= 0 && seg_a + lr >= first_moved) out[d * kRowVec + (q & 15)] = rows[q];
-            }
 #pragma unroll
             for (int k = 0; k < kRegRows; ++k) {
                 const int lr = rs + k * kGroups + g;
-                if (lr < seg) {
+                if (lr < seg && lr >= skip_local) {
                     const int d = dst_of[lr];
-                    if (d >= 0 && seg_a + lr >= first_moved) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
+                    if (d >= 0) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
+                    const uint4* row = concat_row(p.v_cache, p.new_v, u, seg_a + lr, len, B, N);
+                    ra[k] = row[t]; rb[k] = row[t + 8];
                 }
             }
-        }
-        __syncthreads();   // shared-memory rows are free again
-        // ------------------------------------------------------------ a4: V rows: load all, barrier, store all
-        const int skip_local = first_moved - seg_a;   // local rows below this did not move
-        if (tid == 0) {
-            fence_proxy_async();
-            issue_slice_loads(p.v_cache, p.new_v, u, len, B, N, seg_a, rs, skip_local, rows_sa, mbar_sa);
-        }
+#pragma unroll 1
+            for (int s = 0; s < kTilesPerWarp; ++s) {
+                const int tile = warp + kFusedWarps * s;
+                if (tile >= ntiles) break;
+                if (min(rs, (tile + 1) * kTileRows) <= skip_local) continue;   // no row of the tile moves
 #pragma unroll
-        for (int k = 0; k < kRegRows; ++k) {
-            const int lr = rs + k * kGroups + g;
-            if (lr < seg && lr >= skip_local) {
-                const uint4* row = concat_row(p.v_cache, p.new_v, u, seg_a + lr, len, B, N);
-                ra[k] = row[t]; rb[k] = row[t + 8];
+                for (int it = 0; it < 4; ++it) {
+                    const int lr = tile * kTileRows + it * 4 + sub;
+                    if (lr < rs && lr >= skip_local) {
+                        const int d = dst_of[lr];
+                        if (d >= 0) { out[d * kRowVec + t] = rows[lr * kRowVec + t]; out[d * kRowVec + t + 8] = rows[lr * kRowVec + t + 8]; }
+                    }
+                }
+                // The tile's only readers are this warp's lanes and their reads have returned (the stores
+                // above consumed them), so the copy engine may overwrite it: a write after reads needs
+                // execution order only, no proxy fence.
+                __syncwarp();
+                if (lane == 0) issue_tile(p.v_cache, p.new_v, u, len, B, N, sl, tile, rows_sa, mbar_sa);
             }
         }
-        for (int j = 0; j < nchunks; ++j) {
-            if (min(rs, (j + 1) * kChunkRows) <= skip_local) continue;   // chunk was not loaded
-            mbar_wait(mbar_sa + 8 * j, (parity >> j) & 1u, p.status);
-            parity ^= 1u << j;
+        // ------------------------------------------------------------ a4: V rows out, next unit's K rows in behind them
+#pragma unroll 1
+        for (int s = 0; s < kTilesPerWarp; ++s) {
+            const int tile = warp + kFusedWarps * s;
+            if (tile >= ntiles) break;
+            if (min(rs, (tile + 1) * kTileRows) <= skip_local) continue;   // tile was not loaded
+            mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
+            parity ^= 1u << s;
         }
-        cluster_sync_all();   // (3) every V row of the unit that moves is on chip
+        if (kRegRows > 0) {
+            // The register-resident V rows must have ARRIVED, not merely been requested, before any
+            // peer may overwrite their source: fold them into a value the compiler cannot discard.
+            uint32_t fold = 0;
+#pragma unroll
+            for (int k = 0; k < kRegRows; ++k)
+                fold |= (ra[k].x ^ ra[k].y) ^ (ra[k].z ^ ra[k].w) ^ (rb[k].x ^ rb[k].y) ^ (rb[k].z ^ rb[k].w);
+            if (fold == 0x5bd1e995u && n < 0) atomicExch(p.status, kErrTimeout);   // never true: n > 0
+        }
+        cluster_sync_all();   // (3) every warp of the cluster holds the V rows it is responsible for
         {
             uint4* out = p.v_cache + static_cast<size_t>(u) * N * kRowVec;
-            for (int q = tid; q < rs * kRowVec; q += kFusedThreads) {
-                const int lr = q >> 4, d = dst_of[lr];
-                if (d >= 0 && lr >= skip_local) out[d * kRowVec + (q & 15)] = rows[q];
-            }
 #pragma unroll
             for (int k = 0; k < kRegRows; ++k) {
                 const int lr = rs + k * kGroups + g;
@@ -456,9 +581,30 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                     const int d = dst_of[lr];
                     if (d >= 0) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
                 }
+                if (lr < seg && un < p.U) {   // the next unit's K row takes the registers over
+                    const uint4* row = concat_row(p.k_cache, p.new_k, un, seg_a + lr, len, B, N);
+                    ra[k] = row[t]; rb[k] = row[t + 8];
+                }
+            }
+#pragma unroll 1
+            for (int s = 0; s < kTilesPerWarp; ++s) {
+                const int tile = warp + kFusedWarps * s;
+                if (tile >= ntiles) break;
+                if (min(rs, (tile + 1) * kTileRows) > skip_local) {
+#pragma unroll
+                    for (int it = 0; it < 4; ++it) {
+                        const int lr = tile * kTileRows + it * 4 + sub;
+                        if (lr < rs && lr >= skip_local) {
+                            const int d = dst_of[lr];
+                            if (d >= 0) { out[d * kRowVec + t] = rows[lr * kRowVec + t]; out[d * kRowVec + t + 8] = rows[lr * kRowVec + t + 8]; }
+                        }
+                    }
+                    __syncwarp();
+                }
+                if (lane == 0 && un < p.U) issue_tile(p.k_cache, p.new_k, un, len, B, N, sl, tile, rows_sa, mbar_sa);
             }
         }
-        __syncthreads();   // rows / dst_of are free for the next unit
+        __syncthreads();   // dst_of is free for the next unit's reduction scratch
     }
     cluster_sync_all();   // no CTA leaves while a peer may still address its shared memory
 }

@@ -42,6 +42,7 @@ struct keydiff_ctx {
     int fused_nkeys = 0;        // fused path: key-table capacity
     int fused_smem_bytes = 0;
     int fused_max_clusters = 0; // co-resident clusters (grid = min(U, this) * cluster)
+    int fused_reg_rows = 0;     // kernel instance: rows per row group kept in registers
     float eps = kDefaultEps;
     // device scratch
     float* partial = nullptr;         // [U][splits][128]
@@ -75,30 +76,46 @@ int check_step_args(const keydiff_ctx* ctx, const void* k_cache, const void* v_c
     return KEYDIFF_OK;
 }
 
+using FusedKernel = void (*)(kd::FusedParams);
+
+// Kernel instance for `reg_rows` register-resident rows per row group (rounded up to one that is built).
+FusedKernel fused_instance(int reg_rows, int* built) {
+    using namespace kd;
+    if (reg_rows <= 0) { *built = 0; return fused_evict_kernel<0>; }
+    if (reg_rows <= 2) { *built = 2; return fused_evict_kernel<2>; }
+    if (reg_rows <= 4) { *built = 4; return fused_evict_kernel<4>; }
+    if (reg_rows <= 5) { *built = 5; return fused_evict_kernel<5>; }
+    *built = 6; return fused_evict_kernel<6>;
+}
+
 // Choose the cluster size and shared-memory split of the fused kernel for units of up to nmax
 // rows; returns false if no cluster can hold a unit on chip.
 bool plan_fused(keydiff_ctx* c, int sm_count) {
     using namespace kd;
-    const int nkeys = (c->nmax + 31) & ~31;
-    int chosen = 0, chosen_rows = 0;
-    for (int C = 1; C <= 16; C *= 2) {
-        const int per_cta = (c->nmax + C - 1) / C;
-        int sr = kMaxChunks * kChunkRows;
-        while (sr > 0 && fused_layout(sr, nkeys).total > kSmemLimit) sr -= kChunkRows;
+    int chosen = 0, chosen_rows = 0, chosen_keys = 0, chosen_per = 0;
+    for (int C = 1; C <= kMaxCluster; C *= 2) {
+        const int per_cta = ((c->nmax + C - 1) / C + 3) & ~3;        // slices are multiples of 4 rows
+        const int nkeys = C * per_cta;
+        int sr = std::min(kMaxTiles * kTileRows, (per_cta + kTileRows - 1) / kTileRows * kTileRows);
+        while (sr > 0 && fused_layout(sr, nkeys, C).total > kSmemLimit) sr -= kTileRows;
         if (sr <= 0) return false;                                   // the key table alone does not fit
-        if (sr + kRegRows * kGroups < per_cta) continue;             // slice too long for this cluster size
+        if (sr + kMaxRegRows * kGroups < per_cta) continue;          // slice too long for this cluster size
         // small jobs: spread a unit over more SMs while the whole grid still fits the device
         if (chosen == 0 || (C <= 8 && c->U * C <= sm_count)) {
             chosen = C;
-            chosen_rows = std::min(sr, (per_cta + kChunkRows - 1) / kChunkRows * kChunkRows);
+            chosen_rows = sr;
+            chosen_keys = nkeys;
+            chosen_per = per_cta;
         }
         if (C * 2 > 8 && chosen != 0) break;
     }
     if (chosen == 0) return false;
-    const FusedLayout L = fused_layout(chosen_rows, nkeys);
-    if (cudaFuncSetAttribute(fused_evict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess) return false;
+    const FusedLayout L = fused_layout(chosen_rows, chosen_keys, chosen);
+    int reg_rows = 0;
+    const FusedKernel kern = fused_instance((std::max(0, chosen_per - chosen_rows) + kGroups - 1) / kGroups, &reg_rows);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess) return false;
     if (chosen > 8 &&
-        cudaFuncSetAttribute(fused_evict_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return false;
+        cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return false;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(chosen * sm_count);
     cfg.blockDim = dim3(kFusedThreads);
@@ -108,15 +125,16 @@ bool plan_fused(keydiff_ctx* c, int sm_count) {
     attr[0].val.clusterDim.x = chosen; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     int max_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&max_clusters, fused_evict_kernel, &cfg) != cudaSuccess || max_clusters < 1) {
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg) != cudaSuccess || max_clusters < 1) {
         cudaGetLastError();
         return false;
     }
     c->cluster = chosen;
     c->fused_smem_rows = chosen_rows;
-    c->fused_nkeys = nkeys;
+    c->fused_nkeys = chosen_keys;
     c->fused_smem_bytes = L.total;
     c->fused_max_clusters = max_clusters;
+    c->fused_reg_rows = reg_rows;
     return true;
 }
 
@@ -126,12 +144,21 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     p.k_cache = kc; p.v_cache = vc; p.new_k = nk; p.new_v = nv;
     p.len = c->len; p.B = B; p.N = c->cfg.budget; p.U = c->U; p.eps = c->eps;
     p.cluster = c->cluster;
-    p.rows_per_cta = (c->len + B + c->cluster - 1) / c->cluster;
+    p.rows_per_cta = ((c->len + B + c->cluster - 1) / c->cluster + 3) & ~3;
     p.smem_rows = c->fused_smem_rows; p.nkeys = c->fused_nkeys; p.nmax = c->nmax;
     p.scores = c->scores; p.kept_idx = c->kept_idx; p.first_evicted = c->first_evicted;
     p.moved_rows = c->moved_rows; p.status = c->status;
+    const int nclusters = std::min(c->U, c->fused_max_clusters);
+    // Start-up stagger: one unit's estimated duration spread evenly over the co-resident clusters.
+    // A unit moves 4 slices (K in, K out, V in, V out) per SM at roughly 45 GB/s per SM when the other
+    // SMs are busy too, plus a few microseconds of arithmetic and barriers.
+    p.stagger_ns = 0;
+    if (nclusters > 1 && c->U > nclusters) {
+        const double unit_ns = 4.0 * p.rows_per_cta * kRowBytes / 45.0 + 8000.0;
+        p.stagger_ns = static_cast<unsigned>(unit_ns / nclusters);
+    }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(std::min(c->U, c->fused_max_clusters) * c->cluster);
+    cfg.gridDim = dim3(nclusters * c->cluster);
     cfg.blockDim = dim3(kFusedThreads);
     cfg.dynamicSmemBytes = c->fused_smem_bytes;
     cfg.stream = st;
@@ -139,7 +166,8 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = c->cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    KD_CUDA(cudaLaunchKernelEx(&cfg, fused_evict_kernel, p));
+    int built = 0;
+    KD_CUDA(cudaLaunchKernelEx(&cfg, fused_instance(c->fused_reg_rows, &built), p));
     return KEYDIFF_OK;
 }
 
