@@ -88,54 +88,62 @@ FusedKernel fused_instance(int reg_rows, int* built) {
     *built = 6; return fused_evict_kernel<6>;
 }
 
+// Co-resident clusters of `C` CTAs of the fused kernel instance `kern` with `smem` bytes each.
+int max_active_clusters(FusedKernel kern, int C, int smem, int sm_count) {
+    using namespace kd;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return 0;
+    if (C > 8 && cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(C * sm_count);
+    cfg.blockDim = dim3(kFusedThreads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
+}
+
 // Choose the cluster size and shared-memory split of the fused kernel for units of up to nmax
-// rows; returns false if no cluster can hold a unit on chip.
+// rows; returns false if no cluster can hold a unit on chip.  Every cluster size from 1 to 16 is
+// tried: how many clusters the device holds at once depends on how the SMs are grouped (on a B200
+// 15 clusters fit both at 8 and at 9 CTAs, i.e. 120 or 135 SMs), and the estimated step time
+//   ceil(U / clusters) * (fixed cost per unit + cost per slice row * slice rows)
+// picks the winner (constants from per-phase timings of the kernel on a B200).
 bool plan_fused(keydiff_ctx* c, int sm_count) {
     using namespace kd;
-    int chosen = 0, chosen_rows = 0, chosen_keys = 0, chosen_per = 0;
-    for (int C = 1; C <= kMaxCluster; C *= 2) {
+    constexpr double kUnitFixedUs = 10.3, kRowUs = 0.0202;
+    int forced = 0;
+    if (const char* env = std::getenv("KEYDIFF_CLUSTER_SIZE")) forced = std::atoi(env);   // tuning aid
+    double best = 0.0;
+    bool found = false;
+    for (int C = 1; C <= kMaxCluster; ++C) {
+        if (forced > 0 && C != forced) continue;
         const int per_cta = ((c->nmax + C - 1) / C + 3) & ~3;        // slices are multiples of 4 rows
         const int nkeys = C * per_cta;
         int sr = std::min(kMaxTiles * kTileRows, (per_cta + kTileRows - 1) / kTileRows * kTileRows);
         while (sr > 0 && fused_layout(sr, nkeys, C).total > kSmemLimit) sr -= kTileRows;
-        if (sr <= 0) return false;                                   // the key table alone does not fit
+        if (sr <= 0) break;                                          // the key table alone does not fit
         if (sr + kMaxRegRows * kGroups < per_cta) continue;          // slice too long for this cluster size
-        // small jobs: spread a unit over more SMs while the whole grid still fits the device
-        if (chosen == 0 || (C <= 8 && c->U * C <= sm_count)) {
-            chosen = C;
-            chosen_rows = sr;
-            chosen_keys = nkeys;
-            chosen_per = per_cta;
+        const int smem = fused_layout(sr, nkeys, C).total;
+        int reg_rows = 0;
+        const FusedKernel kern = fused_instance((std::max(0, per_cta - sr) + kGroups - 1) / kGroups, &reg_rows);
+        const int clusters = max_active_clusters(kern, C, smem, sm_count);
+        if (clusters < 1) continue;
+        const int used = std::min(c->U, clusters);
+        const double est = static_cast<double>((c->U + used - 1) / used) * (kUnitFixedUs + kRowUs * per_cta);
+        if (!found || est < 0.95 * best) {   // a larger cluster has to pay for its extra barrier traffic
+            found = true; best = est;
+            c->cluster = C; c->fused_smem_rows = sr; c->fused_nkeys = nkeys; c->fused_smem_bytes = smem;
+            c->fused_max_clusters = clusters; c->fused_reg_rows = reg_rows;
         }
-        if (C * 2 > 8 && chosen != 0) break;
     }
-    if (chosen == 0) return false;
-    const FusedLayout L = fused_layout(chosen_rows, chosen_keys, chosen);
-    int reg_rows = 0;
-    const FusedKernel kern = fused_instance((std::max(0, chosen_per - chosen_rows) + kGroups - 1) / kGroups, &reg_rows);
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L.total) != cudaSuccess) return false;
-    if (chosen > 8 &&
-        cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return false;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(chosen * sm_count);
-    cfg.blockDim = dim3(kFusedThreads);
-    cfg.dynamicSmemBytes = L.total;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = chosen; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    int max_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&max_clusters, kern, &cfg) != cudaSuccess || max_clusters < 1) {
-        cudaGetLastError();
-        return false;
-    }
-    c->cluster = chosen;
-    c->fused_smem_rows = chosen_rows;
-    c->fused_nkeys = chosen_keys;
-    c->fused_smem_bytes = L.total;
-    c->fused_max_clusters = max_clusters;
-    c->fused_reg_rows = reg_rows;
-    return true;
+    if (!found) return false;
+    // the attributes of the chosen instance (the loop may have left another size's values behind)
+    int built = 0;
+    return max_active_clusters(fused_instance(c->fused_reg_rows, &built), c->cluster, c->fused_smem_bytes, sm_count) >= 1;
 }
 
 int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const uint4* nv, int B, cudaStream_t st) {
