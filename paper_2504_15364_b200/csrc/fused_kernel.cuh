@@ -12,10 +12,13 @@
 //               of e_i goes into this CTA's part of the key table, the part is then pushed to
 //               all peers with 128-bit DSMEM stores and one cluster barrier completes the table
 //               everywhere (App. B.1, expr. 2).  fp32 scores go to global scratch, coalesced.
-//   a3 select   every CTA finds the N-th largest key of the full table locally: a 2048-bin
-//               histogram over a monotone fixed-point image of e, then an exact rank among the
-//               few keys of the threshold bin; a 4x8-bit radix select is the fallback when that
-//               bin is crowded.  Ties keep the older token (Eq. efficient-keydiff, topk).
+//   a3 select   every CTA selects on its own copy of the table.  Only E = n - N keys go, so the work
+//               is at the low end: a 2048-bin histogram over the unit's own key range, the bin
+//               where the running count from below reaches E, a bitmap of the tokens under that
+//               bin, an exact rank among the bin's own few keys.  Crowded bins (many equal scores)
+//               and large units fall back to a histogram over a fixed-point image of e with an
+//               exact rank or a 4x8-bit radix select.  Ties keep the older token (Eq.
+//               efficient-keydiff, topk).
 //   a4 compact  an ordered scan gives every kept row its destination; the rows then leave the
 //               chip tile by tile, and each shared-memory tile is refilled as soon as it has
 //               been written out: K stores hand their tile to the V load of the same rows, V
@@ -47,6 +50,8 @@ constexpr int kMaxRegRows = 6;                          // + up to 6 rows per gr
 constexpr int kBins = 2048;                             // histogram over e in [-1, 1]
 constexpr int kCandCap = kFusedThreads;                 // exact-rank stage handles this many candidates
 constexpr int kMaxCluster = 16;
+constexpr int kFastKeys = 17;                           // fast select: keys per thread held in registers (n <= 8704)
+constexpr int kFastCandCap = 192;                       // fast select: keys of the threshold bin ranked exactly
 constexpr int kSmemLimit = 232448;                      // opt-in shared memory per CTA on sm_100
 constexpr int kErrTimeout = -6;                         // KEYDIFF_ERR_TIMEOUT
 constexpr uint32_t kWaitSpins = 1u << 24;               // bound of every mbarrier wait
@@ -216,6 +221,42 @@ __device__ __forceinline__ uint32_t row_a2(const uint4& a, const uint4& b, const
     return order_key(e == 0.f ? 0.f : e);
 }
 
+// Search in the 2048-bin histogram from the low end, two levels and one CTA barrier: warp w sums bins
+// [128w, 128w+128); every warp then finds the owner warp from the 16 totals and scans that warp's 128
+// bins (4 per lane).  Returns (smallest bin whose inclusive running count reaches E) << 16 | count
+// strictly below it, or -1 if the total stays under E.  All threads must call; the result is uniform.
+__device__ __forceinline__ int find_crossing(const int* h, int E, int lane, int warp, int* wtot) {
+    const int4 v = reinterpret_cast<const int4*>(h)[32 * warp + lane];
+    int s = (v.x + v.y) + (v.z + v.w);
+    s = __reduce_add_sync(0xffffffffu, s);
+    if (lane == 0) wtot[warp] = s;
+    __syncthreads();
+    const int t = lane < kFusedWarps ? wtot[lane] : 0;
+    int incl = t;
+#pragma unroll
+    for (int o = 1; o < 16; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += x; }
+    const unsigned hit = __ballot_sync(0xffffffffu, lane < kFusedWarps && incl - t < E && E <= incl);
+    if (hit == 0) return -1;
+    const int W = __ffs(hit) - 1;
+    const int base = __shfl_sync(0xffffffffu, incl - t, W);
+    const int4 c = reinterpret_cast<const int4*>(h)[32 * W + lane];
+    const int c4 = (c.x + c.y) + (c.z + c.w);
+    int incl2 = c4;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, incl2, o); if (lane >= o) incl2 += x; }
+    const unsigned hit2 = __ballot_sync(0xffffffffu, base + incl2 >= E);
+    const int J = __ffs(hit2) - 1;          // hit2 != 0: warp W's range crosses E
+    int before = base + __shfl_sync(0xffffffffu, incl2 - c4, J);
+    const int cx = __shfl_sync(0xffffffffu, c.x, J), cy = __shfl_sync(0xffffffffu, c.y, J), cz = __shfl_sync(0xffffffffu, c.z, J);
+    const int bin = 128 * W + 4 * J;
+    if (before + cx >= E) return (bin << 16) | before;
+    before += cx;
+    if (before + cy >= E) return ((bin + 1) << 16) | before;
+    before += cy;
+    if (before + cz >= E) return ((bin + 2) << 16) | before;
+    return ((bin + 3) << 16) | (before + cz);
+}
+
 // Exact top-N over the whole key table by one CTA (every CTA of the cluster runs it on its own
 // copy and gets the same answer): 2048-bin histogram, exact rank inside the threshold bin, radix
 // select when that bin is crowded; then an ordered scan gives every kept row of this CTA's slice
@@ -342,8 +383,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = tid >> 3, t = tid & 7, sub = lane >> 3;
     const int crank = static_cast<int>(cluster_ctarank());
     const int cluster_id = blockIdx.x / C, nclusters = gridDim.x / C;
-    const int len = p.len, B = p.B, N = p.N, n = len + B;
+    const int len = p.len, B = p.B, N = p.N, n = len + B, E = n - N;   // E tokens are evicted
     const float inv_eps = 1.0f / p.eps;
+    // fast select: evicted-token bitmap, its per-word prefix and the threshold bin's keys share `xchg`
+    const int nwords = (n + 31) >> 5;
+    uint32_t* bitmap = reinterpret_cast<uint32_t*>(smem + L.xchg);
+    int* wlocal = reinterpret_cast<int*>(smem + L.xchg) + nwords;
+    uint32_t* fcand_key = reinterpret_cast<uint32_t*>(smem + L.xchg) + 2 * nwords;
+    int* fcand_idx = reinterpret_cast<int*>(smem + L.xchg) + 2 * nwords + kFastCandCap;
+    const bool fast_ok = n <= kFastKeys * kFusedThreads &&
+                         2 * nwords + 2 * kFastCandCap <= max(C * kHeadDim, 2 * kCandCap);   // uniform over the grid
     Slice sl;
     sl.seg_a = min(n, crank * p.rows_per_cta);
     sl.seg = min(n, sl.seg_a + p.rows_per_cta) - sl.seg_a;
@@ -505,10 +554,127 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         {
             float* sc = p.scores + static_cast<size_t>(u) * p.nmax + seg_a;   // fp32 scores to global scratch, coalesced
             for (int lr = tid; lr < seg; lr += kFusedThreads) sc[lr] = key_score(keys[seg_a + lr]);
+            if (fast_ok) {
+                for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;          // `red` is dead
+                for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;   // the partials are dead
+                if (tid == 0) { misc[0] = 0; misc[1] = n; }
+            }
         }
         cluster_wait();       // (2) the key table of every CTA holds all n keys
         // ------------------------------------------------------------ a3 + plan: who is evicted, where every kept row goes
-        full_select_plan(keys, n, N, seg_a, seg_b, hist, cand_key, cand_idx, dst_of, sel, misc);
+        bool planned = false;
+        if (fast_ok) {
+            // Only E keys go, so the work is at the low end.  Thread t keeps the keys of tokens t, t+512, ...
+            // in registers; the 2048 bins are spread over the low end of the unit's own key range (from the
+            // smallest key to a bound on the E-th smallest; monotone in the key, which is all selection needs); the
+            // tokens under the threshold bin go straight into a bitmap, the bin's own few keys are ranked
+            // exactly, and prefix counts over the bitmap give every kept row of the slice its destination.
+            uint32_t* wmin = reinterpret_cast<uint32_t*>(sel.hist);          // (sel.hist is radix-select scratch)
+            uint32_t* wmax = reinterpret_cast<uint32_t*>(sel.hist) + kFusedWarps;
+            int* wbase = sel.hist + 2 * kFusedWarps;
+            const int cnt = (n - tid + kFusedThreads - 1) / kFusedThreads;
+            uint32_t kk[kFastKeys];
+#pragma unroll
+            for (int j = 0; j < kFastKeys; ++j) kk[j] = j < cnt ? keys[tid + j * kFusedThreads] : 0xffffffffu;
+            {
+                uint32_t lo = 0xffffffffu, hi = 0u;
+#pragma unroll
+                for (int j = 0; j < kFastKeys; ++j) { lo = min(lo, kk[j]); if (j < cnt) hi = max(hi, kk[j]); }
+                // The E-th smallest key is at most the largest of any E distinct keys.  When at least E
+                // threads hold keys, the thread minima are such keys, so the largest thread minimum bounds
+                // it; otherwise the largest key does.  Keys above the bound share the top bin.
+                const uint32_t cut = (n >= kFusedThreads && E <= kFusedThreads) ? lo : hi;
+                const uint32_t wlo = __reduce_min_sync(0xffffffffu, lo);
+                const uint32_t wcut = __reduce_max_sync(0xffffffffu, cnt > 0 ? cut : 0u);
+                if (lane == 0) { wmin[warp] = wlo; wmax[warp] = wcut; }
+            }
+            __syncthreads();
+            uint32_t kmin, kcut, shift;
+            {
+                const uint32_t lo = lane < kFusedWarps ? wmin[lane] : 0xffffffffu, hi = lane < kFusedWarps ? wmax[lane] : 0u;
+                kmin = __reduce_min_sync(0xffffffffu, lo);
+                kcut = __reduce_max_sync(0xffffffffu, hi);
+                const int bits = 32 - __clz(kcut - kmin);   // significant bits of the range [kmin, kcut]
+                shift = bits > 11 ? bits - 11 : 0;          // (key - kmin) >> shift < 2048 inside the range
+            }
+            // bin of a key: linear in the key over [kmin, kcut] (bins 0..2046), 2047 above; monotone
+            auto bin_of = [kmin, kcut, shift](uint32_t k) { return k <= kcut ? min((k - kmin) >> shift, 2046u) : 2047u; };
+#pragma unroll
+            for (int j = 0; j < kFastKeys; ++j) if (j < cnt) atomicAdd(&hist[bin_of(kk[j])], 1);
+            __syncthreads();
+            const int packed = find_crossing(hist, E, lane, warp, sel.warp_eq);
+            const uint32_t bstar = static_cast<uint32_t>(packed >> 16);
+            const int need = E - (packed & 0xffff);   // this many keys of the threshold bin go
+            unsigned m_below = 0, m_in = 0;           // bit j: this thread's j-th key is below / inside the bin
+#pragma unroll
+            for (int j = 0; j < kFastKeys; ++j) {
+                const uint32_t b = bin_of(kk[j]);
+                m_below |= (j < cnt && b < bstar) ? 1u << j : 0u;
+                m_in |= (j < cnt && b == bstar) ? 1u << j : 0u;
+            }
+            if (packed >= 0 && (m_below | m_in)) {
+                int first = n;
+                for (unsigned m = m_below; m; m &= m - 1) {
+                    const int i = tid + (__ffs(m) - 1) * kFusedThreads;
+                    atomicOr(&bitmap[i >> 5], 1u << (i & 31));
+                    first = min(first, i);
+                }
+                for (unsigned m = m_in; m; m &= m - 1) {
+                    const int i = tid + (__ffs(m) - 1) * kFusedThreads;
+                    const int slot = atomicAdd(&misc[0], 1);
+                    if (slot < kFastCandCap) { fcand_key[slot] = keys[i]; fcand_idx[slot] = i; }
+                }
+                if (first < n) atomicMin(&misc[1], first);
+            }
+            __syncthreads();
+            const int ncand = misc[0];
+            if (packed >= 0 && ncand <= kFastCandCap) {   // uniform: every thread sees the same values
+                // Eviction order is the reverse of the keep order: key ascending, index descending.
+                int wfirst = n;
+                for (int c = warp; c < ncand; c += kFusedWarps) {
+                    const uint32_t mk = fcand_key[c];
+                    const int mi = fcand_idx[c];
+                    int rank = 0;
+                    for (int q = lane; q < ncand; q += 32) {
+                        const uint32_t ok = fcand_key[q];
+                        rank += (ok < mk) || (ok == mk && fcand_idx[q] > mi);
+                    }
+                    rank = __reduce_add_sync(0xffffffffu, rank);
+                    if (lane == 0 && rank < need) { atomicOr(&bitmap[mi >> 5], 1u << (mi & 31)); wfirst = min(wfirst, mi); }
+                }
+                if (lane == 0 && wfirst < n) atomicMin(&misc[1], wfirst);
+                __syncthreads();
+                {
+                    // evicted tokens before each word of the bitmap: one word per thread (nwords <= 512)
+                    const int pc = tid < nwords ? __popc(bitmap[tid]) : 0;
+                    int incl = pc;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= o) incl += v;
+                    }
+                    if (tid < nwords) wlocal[tid] = incl - pc;
+                    if (lane == 31) sel.warp_gt[warp] = incl;
+                }
+                __syncthreads();
+                if (warp == 0) {
+                    const int t2 = lane < kFusedWarps ? sel.warp_gt[lane] : 0;
+                    int incl = t2;
+#pragma unroll
+                    for (int o = 1; o < 16; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
+                    if (lane < kFusedWarps) wbase[lane] = incl - t2;
+                }
+                __syncthreads();
+                for (int lr = tid; lr < seg; lr += kFusedThreads) {
+                    const int i = seg_a + lr, w = i >> 5;
+                    const uint32_t wd = bitmap[w], bit = 1u << (i & 31);
+                    dst_of[lr] = (wd & bit) ? -1 : i - (wbase[w >> 5] + wlocal[w] + __popc(wd & (bit - 1)));
+                }
+                __syncthreads();
+                planned = true;
+            }
+        }
+        if (!planned) full_select_plan(keys, n, N, seg_a, seg_b, hist, cand_key, cand_idx, dst_of, sel, misc);
         const int first_evicted = misc[1];
         const int first_moved = min(first_evicted, len);   // block rows always move into the cache
         const int skip_local = first_moved - seg_a;        // local rows below this keep their place
