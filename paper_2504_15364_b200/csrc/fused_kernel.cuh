@@ -67,7 +67,7 @@ __host__ __device__ inline FusedLayout fused_layout(int smem_rows, int nkeys, in
     int off = 0;
     auto take = [&off](int bytes) { const int o = off; off += (bytes + 127) & ~127; return o; };
     L.rows = take(smem_rows * kRowBytes);
-    L.keys = take(nkeys * 4);
+    L.keys = take(nkeys * 4 > kBins * 4 ? nkeys * 4 : kBins * 4);   // also 8 KB of reduction scratch while the table is dead
     L.work = take(kBins * 4);   // warp-reduction scratch / histogram / destination table (never live together)
     L.xchg = take(C * kHeadDim * 4 > 2 * kCandCap * 4 ? C * kHeadDim * 4 : 2 * kCandCap * 4);   // anchor partials [C][128] / candidates
     L.sel = take(static_cast<int>(sizeof(SelectSmem)));
@@ -90,6 +90,10 @@ struct FusedParams {
     unsigned stagger_ns; // cluster c starts c * stagger_ns late (see the kernel)
     float* scores; int32_t* kept_idx; int32_t* first_evicted;
     unsigned long long* moved_rows; int32_t* status;
+    // running anchor (see the kernel): sum of k/||k|| over the cached rows as of the previous step
+    // = anchor_in[u][c] + sum over CTA ranks r of anchor_delta[u][r][c]; this step writes anchor_out and
+    // new deltas
+    const double* anchor_in; double* anchor_out; float* anchor_delta;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -211,6 +215,15 @@ __device__ __forceinline__ float row_a1(const uint4& a, const uint4& b, bool val
 #pragma unroll
     for (int p = 0; p < 8; ++p) acc[p] = __ffma2_rn(x[p], inv2, acc[p]);
     return approx_sqrt(ss);
+}
+// Steps a1 + a2 for one row when the anchor is known beforehand: norm and dot product in one pass.
+__device__ __forceinline__ uint32_t row_score(const uint4& a, const uint4& b, const float2 (&w)[8], float m, float eps) {
+    float2 x[8];
+    unpack_pairs(a, b, x);
+    const float r = approx_sqrt(pairs_sumsq(x));
+    const float dot = pairs_dot(x, w);
+    const float e = -(dot * approx_rcp(fmaxf(m * r, eps)));
+    return order_key(e == 0.f ? 0.f : e);
 }
 // Step a2 for one row: orderable key of e = -(mu.k)/max(||mu|| ||k||, eps), -0 mapped to +0.
 __device__ __forceinline__ uint32_t row_a2(const uint4& a, const uint4& b, const float2 (&w)[8], float m, float r, float eps) {
@@ -361,7 +374,17 @@ __device__ __noinline__ void full_select_plan(const uint32_t* keys, int n, int N
 
 // kRegRows = rows per row group that live in registers (the host picks the smallest instance that
 // holds a slice together with the shared-memory rows).
-template <int kRegRows>
+//
+// kOnePass: the anchor is known before the keys are read.  The library keeps, per unit, the sum of
+// k/||k|| over the rows in the cache (App. B.1, expr. 1, split over time): a step's sum over its n rows
+// is that running sum plus the sum over the B block rows, so only the block has to be normalised
+// before scoring, norm and dot product of a row are taken in one pass while the tiles land, and the
+// first cluster barrier, the anchor exchange and the second pass over the rows disappear.  Every step
+// (either kind) subtracts the evicted rows' k/||k|| again: each CTA leaves the change it saw in
+// anchor_delta, and the next step folds the deltas into the running sum in double precision, in a
+// fixed order.  kOnePass = false recomputes the anchor from all n rows (first evicting step, after
+// set_len / reset / appends, and periodically to shed rounding drift).
+template <int kRegRows, bool kOnePass>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const FusedParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int C = p.cluster;
@@ -441,6 +464,99 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
 
     for (int u = cluster_id; u < p.U; u += nclusters) {
         const int un = u + nclusters;   // the unit this cluster serves next
+        float block_sum = 0.f;   // tid < 128: channel tid of the block rows' sum of k/||k||
+        if constexpr (kOnePass) {
+        // ------------------------------------------------------------ anchor from the running sum + the block rows
+        {
+            // the running sum and its pending deltas, requested first: they arrive under the block's arithmetic
+            double run = 0.0;
+            float dl[kMaxCluster];
+            if (tid < kHeadDim) {
+                run = p.anchor_in[static_cast<size_t>(u) * kHeadDim + tid];
+#pragma unroll
+                for (int c = 0; c < kMaxCluster; ++c)
+                    dl[c] = c < C ? p.anchor_delta[(static_cast<size_t>(u) * C + c) * kHeadDim + tid] : 0.f;
+            }
+            float2 acc[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc[q] = make_float2(0.f, 0.f);
+            for (int b0 = 0; b0 < B; b0 += kGroups) {   // every CTA normalises the whole block: no exchange needed
+                const int br = b0 + g;                   // (same trip count in every lane: row_a1 shuffles)
+                uint4 a = make_uint4(0, 0, 0, 0), b = a;
+                if (br < B) {
+                    const uint4* row = p.new_k + (static_cast<size_t>(u) * B + br) * kRowVec;
+                    a = row[t]; b = row[t + 8];
+                }
+                row_a1(a, b, br < B, inv_eps, acc);
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                float2 v = acc[q];
+                v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
+                v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
+                acc[q] = v;
+            }
+            if (lane < 8) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<float2*>(&red[warp * kHeadDim + lane_channel(t, 2 * q)]) = acc[q];
+            }
+            __syncthreads();
+            if (tid < kHeadDim) {
+#pragma unroll
+                for (int w = 0; w < kFusedWarps; ++w) block_sum += red[w * kHeadDim + tid];
+                double a = run;
+#pragma unroll
+                for (int c = 0; c < kMaxCluster; ++c) a += static_cast<double>(dl[c]);   // rank order; absent ranks add 0
+                if (crank == 0) p.anchor_out[static_cast<size_t>(u) * kHeadDim + tid] = a;   // the cached rows' sum, folded
+                mu_sh[tid] = static_cast<float>((a + static_cast<double>(block_sum)) / static_cast<double>(n));
+            }
+            __syncthreads();
+        }
+        // ------------------------------------------------------------ a1 + a2 in one pass: keys of this slice
+        {
+            float2 w[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) w[q] = *reinterpret_cast<const float2*>(&mu_sh[lane_channel(t, 2 * q)]);
+            float m;   // ||mu||, computed by every warp in the same order
+            {
+                const float4 c4 = reinterpret_cast<const float4*>(mu_sh)[lane];
+                float v = fmaf(c4.w, c4.w, fmaf(c4.z, c4.z, fmaf(c4.y, c4.y, c4.x * c4.x)));
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                m = sqrtf(v);
+            }
+#pragma unroll 1
+            for (int s = 0; s < kTilesPerWarp; ++s) {
+                const int tile = warp + kFusedWarps * s;
+                if (tile >= ntiles) break;
+                mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
+                parity ^= 1u << s;
+#pragma unroll 1
+                for (int half = 0; half < 2; ++half) {
+                    uint4 a[2], b[2];
+#pragma unroll
+                    for (int it = 0; it < 2; ++it) {
+                        const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
+                        a[it] = make_uint4(0, 0, 0, 0); b[it] = a[it];
+                        if (lr < rs) { a[it] = rows[lr * kRowVec + t]; b[it] = rows[lr * kRowVec + t + 8]; }
+                    }
+#pragma unroll
+                    for (int it = 0; it < 2; ++it) {
+                        const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
+                        const uint32_t key = row_score(a[it], b[it], w, m, p.eps);
+                        if (lr < rs && t == 0) keys[seg_a + lr] = key;
+                    }
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < kRegRows; ++k) {
+                const uint32_t key = row_score(ra[k], rb[k], w, m, p.eps);
+                const int lr = rs + k * kGroups + g;
+                if (lr < seg && t == 0) keys[seg_a + lr] = key;
+            }
+        }
+        } else {
         // ------------------------------------------------------------ a1: norms and anchor partial
         float2 acc[8];
 #pragma unroll
@@ -496,6 +612,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             float s = 0.f;
             for (int c = 0; c < C; ++c) s += partials[c * kHeadDim + tid];   // rank order: same bits in every CTA
             mu_sh[tid] = s / static_cast<float>(n);
+            if (crank == 0) p.anchor_out[static_cast<size_t>(u) * kHeadDim + tid] = static_cast<double>(s);   // sum over all n rows
         }
         __syncthreads();
         // ------------------------------------------------------------ a2: keys of this slice into the table
@@ -540,6 +657,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 if (lr < seg && t == 0) keys[seg_a + lr] = key;
             }
         }
+        }   // kOnePass
         __syncthreads();
         {
             // this slice's keys -> every peer's table (128-bit DSMEM stores)
@@ -689,12 +807,23 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         // ------------------------------------------------------------ a4: K rows out, V rows in behind them
         {
             uint4* out = p.k_cache + static_cast<size_t>(u) * N * kRowVec;
+            float2 gone[8];   // sum of k/||k|| over this thread's share of the evicted rows (for the running anchor)
+#pragma unroll
+            for (int q = 0; q < 8; ++q) gone[q] = make_float2(0.f, 0.f);
+            if (kOnePass && crank == 0 && un < p.U) {   // the next unit's block rows towards L2: every CTA reads them first thing
+                const char* nb = reinterpret_cast<const char*>(p.new_k + static_cast<size_t>(un) * B * kRowVec);
+                for (int o = tid * 128; o < B * kRowBytes; o += kFusedThreads * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(nb + o));
+            }
+            // (row_a1 shuffles inside each row group, so the whole warp enters it together: the vote is
+            // warp-wide, the row's own flag only decides whether it contributes)
 #pragma unroll
             for (int k = 0; k < kRegRows; ++k) {
                 const int lr = rs + k * kGroups + g;
-                if (lr < seg && lr >= skip_local) {
-                    const int d = dst_of[lr];
-                    if (d >= 0) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
+                const bool vis = lr < seg && lr >= skip_local;
+                const int d = vis ? dst_of[lr] : 0;
+                if (vis && d >= 0) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
+                if (__any_sync(0xffffffffu, vis && d < 0)) row_a1(ra[k], rb[k], vis && d < 0, inv_eps, gone);
+                if (vis) {
                     const uint4* row = concat_row(p.v_cache, p.new_v, u, seg_a + lr, len, B, N);
                     ra[k] = row[t]; rb[k] = row[t + 8];
                 }
@@ -704,19 +833,43 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 const int tile = warp + kFusedWarps * s;
                 if (tile >= ntiles) break;
                 if (min(rs, (tile + 1) * kTileRows) <= skip_local) continue;   // no row of the tile moves
-#pragma unroll
+#pragma unroll 1
                 for (int it = 0; it < 4; ++it) {
                     const int lr = tile * kTileRows + it * 4 + sub;
-                    if (lr < rs && lr >= skip_local) {
-                        const int d = dst_of[lr];
-                        if (d >= 0) { out[d * kRowVec + t] = rows[lr * kRowVec + t]; out[d * kRowVec + t + 8] = rows[lr * kRowVec + t + 8]; }
-                    }
+                    const bool vis = lr < rs && lr >= skip_local;
+                    const int d = vis ? dst_of[lr] : 0;
+                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
+                    if (vis) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
+                    if (vis && d >= 0) { out[d * kRowVec + t] = a; out[d * kRowVec + t + 8] = b; }
+                    if (__any_sync(0xffffffffu, vis && d < 0)) row_a1(a, b, vis && d < 0, inv_eps, gone);
                 }
                 // The tile's only readers are this warp's lanes and their reads have returned (the stores
                 // above consumed them), so the copy engine may overwrite it: a write after reads needs
                 // execution order only, no proxy fence.
                 __syncwarp();
                 if (lane == 0) issue_tile(p.v_cache, p.new_v, u, len, B, N, sl, tile, rows_sa, mbar_sa);
+            }
+            // what this CTA saw leave (and, on rank 0 of a one-pass step, the block that came in): its delta
+            // to the running sum.  The key table is dead until the next unit: 8 KB of it serve as scratch.
+            float* red2 = reinterpret_cast<float*>(keys);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                float2 v = gone[q];
+                v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
+                v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
+                gone[q] = v;
+            }
+            if (lane < 8) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<float2*>(&red2[warp * kHeadDim + lane_channel(t, 2 * q)]) = gone[q];
+            }
+            __syncthreads();
+            if (tid < kHeadDim) {
+                float e = 0.f;
+#pragma unroll
+                for (int w = 0; w < kFusedWarps; ++w) e += red2[w * kHeadDim + tid];
+                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass && crank == 0 ? block_sum : 0.f) - e;
             }
         }
         // ------------------------------------------------------------ a4: V rows out, next unit's K rows in behind them

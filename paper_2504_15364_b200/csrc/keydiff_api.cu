@@ -43,6 +43,13 @@ struct keydiff_ctx {
     int fused_smem_bytes = 0;
     int fused_max_clusters = 0; // co-resident clusters (grid = min(U, this) * cluster)
     int fused_reg_rows = 0;     // kernel instance: rows per row group kept in registers
+    // running anchor of the fused path: sum of k/||k|| over the cached rows, per unit
+    bool incremental = true;    // use it (one-pass kernel) when it is valid
+    bool anchor_valid = false;  // the buffers describe the cache as the last evicting step left it
+    int anchor_par = 0;         // which of the two sum buffers the next step reads
+    int steps_since_full = 0;   // one-pass steps since the anchor was last recomputed from all rows
+    double* anchor_sum[2] = {nullptr, nullptr};   // [U][128]
+    float* anchor_delta = nullptr;                // [U][cluster][128]
     float eps = kDefaultEps;
     // device scratch
     float* partial = nullptr;         // [U][splits][128]
@@ -61,6 +68,7 @@ namespace {
 void free_scratch(keydiff_ctx* c) {
     cudaFree(c->partial); cudaFree(c->norms); cudaFree(c->scores); cudaFree(c->kept_idx);
     cudaFree(c->first_evicted); cudaFree(c->status); cudaFree(c->moved_rows); cudaFree(c->stage_k); cudaFree(c->stage_v);
+    cudaFree(c->anchor_sum[0]); cudaFree(c->anchor_sum[1]); cudaFree(c->anchor_delta);
 }
 
 int check_step_args(const keydiff_ctx* ctx, const void* k_cache, const void* v_cache,
@@ -78,14 +86,19 @@ int check_step_args(const keydiff_ctx* ctx, const void* k_cache, const void* v_c
 
 using FusedKernel = void (*)(kd::FusedParams);
 
-// Kernel instance for `reg_rows` register-resident rows per row group (rounded up to one that is built).
-FusedKernel fused_instance(int reg_rows, int* built) {
+// Kernel instance for `reg_rows` register-resident rows per row group (rounded up to one that is
+// built); one_pass = the variant that takes the anchor from the running sum.
+template <bool kOnePass>
+FusedKernel fused_instance_of(int reg_rows, int* built) {
     using namespace kd;
-    if (reg_rows <= 0) { *built = 0; return fused_evict_kernel<0>; }
-    if (reg_rows <= 2) { *built = 2; return fused_evict_kernel<2>; }
-    if (reg_rows <= 4) { *built = 4; return fused_evict_kernel<4>; }
-    if (reg_rows <= 5) { *built = 5; return fused_evict_kernel<5>; }
-    *built = 6; return fused_evict_kernel<6>;
+    if (reg_rows <= 0) { *built = 0; return fused_evict_kernel<0, kOnePass>; }
+    if (reg_rows <= 2) { *built = 2; return fused_evict_kernel<2, kOnePass>; }
+    if (reg_rows <= 4) { *built = 4; return fused_evict_kernel<4, kOnePass>; }
+    if (reg_rows <= 5) { *built = 5; return fused_evict_kernel<5, kOnePass>; }
+    *built = 6; return fused_evict_kernel<6, kOnePass>;
+}
+FusedKernel fused_instance(int reg_rows, int* built, bool one_pass = false) {
+    return one_pass ? fused_instance_of<true>(reg_rows, built) : fused_instance_of<false>(reg_rows, built);
 }
 
 // Co-resident clusters of `C` CTAs of the fused kernel instance `kern` with `smem` bytes each.
@@ -143,7 +156,8 @@ bool plan_fused(keydiff_ctx* c, int sm_count) {
     if (!found) return false;
     // the attributes of the chosen instance (the loop may have left another size's values behind)
     int built = 0;
-    return max_active_clusters(fused_instance(c->fused_reg_rows, &built), c->cluster, c->fused_smem_bytes, sm_count) >= 1;
+    return max_active_clusters(fused_instance(c->fused_reg_rows, &built, false), c->cluster, c->fused_smem_bytes, sm_count) >= 1 &&
+           max_active_clusters(fused_instance(c->fused_reg_rows, &built, true), c->cluster, c->fused_smem_bytes, sm_count) >= 1;
 }
 
 int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const uint4* nv, int B, cudaStream_t st) {
@@ -156,6 +170,12 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     p.smem_rows = c->fused_smem_rows; p.nkeys = c->fused_nkeys; p.nmax = c->nmax;
     p.scores = c->scores; p.kept_idx = c->kept_idx; p.first_evicted = c->first_evicted;
     p.moved_rows = c->moved_rows; p.status = c->status;
+    // The one-pass kernel needs the running anchor of the cache as it stands; every 1024 steps the
+    // anchor is recomputed from all rows anyway, which sheds whatever rounding drift has built up.
+    const bool one_pass = c->incremental && c->anchor_valid && c->steps_since_full < 1024;
+    p.anchor_in = c->anchor_sum[c->anchor_par];
+    p.anchor_out = c->anchor_sum[c->anchor_par ^ 1];
+    p.anchor_delta = c->anchor_delta;
     const int nclusters = std::min(c->U, c->fused_max_clusters);
     // Start-up stagger: one unit's estimated duration spread evenly over the co-resident clusters.
     // A unit moves 4 slices (K in, K out, V in, V out) per SM at roughly 45 GB/s per SM when the other
@@ -175,7 +195,10 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     attr[0].val.clusterDim.x = c->cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     int built = 0;
-    KD_CUDA(cudaLaunchKernelEx(&cfg, fused_instance(c->fused_reg_rows, &built), p));
+    KD_CUDA(cudaLaunchKernelEx(&cfg, fused_instance(c->fused_reg_rows, &built, one_pass), p));
+    c->anchor_par ^= 1;
+    c->anchor_valid = true;
+    c->steps_since_full = one_pass ? c->steps_since_full + 1 : 0;
     return KEYDIFF_OK;
 }
 
@@ -257,6 +280,13 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
     if (ok && cfg->path != KEYDIFF_PATH_STAGED) {
         if (plan_fused(c, prop.multiProcessorCount)) {
             c->path = KEYDIFF_PATH_FUSED;
+            const size_t sum_bytes = sizeof(double) * U * kd::kHeadDim;
+            ok = cudaMalloc(&c->anchor_sum[0], sum_bytes) == cudaSuccess && cudaMalloc(&c->anchor_sum[1], sum_bytes) == cudaSuccess &&
+                 cudaMalloc(&c->anchor_delta, sizeof(float) * U * c->cluster * kd::kHeadDim) == cudaSuccess &&
+                 cudaMemset(c->anchor_sum[0], 0, sum_bytes) == cudaSuccess && cudaMemset(c->anchor_sum[1], 0, sum_bytes) == cudaSuccess &&
+                 cudaMemset(c->anchor_delta, 0, sizeof(float) * U * c->cluster * kd::kHeadDim) == cudaSuccess &&
+                 cudaDeviceSynchronize() == cudaSuccess;
+            if (const char* env = std::getenv("KEYDIFF_INCREMENTAL")) c->incremental = env[0] != '0';   // tuning aid
         } else if (cfg->path == KEYDIFF_PATH_FUSED) {
             free_scratch(c);
             delete c;
@@ -293,6 +323,7 @@ int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache, const void* ne
         kd::append_kernel<<<grid, threads, 0, st>>>(kc, vc, nk, nv, ctx->len, block_B, N);
         KD_CUDA(cudaGetLastError());
         ctx->len = n;
+        ctx->anchor_valid = false;   // the appended rows are not in the running anchor
         return KEYDIFF_OK;
     }
     const int lrc = ctx->path == KEYDIFF_PATH_FUSED ? launch_fused(ctx, kc, vc, nk, nv, block_B, st)
@@ -346,6 +377,7 @@ int keydiff_destroy(keydiff_ctx* ctx) {
 int keydiff_reset(keydiff_ctx* ctx) {
     if (!ctx) return KEYDIFF_ERR_INVALID_ARG;
     ctx->len = 0;
+    ctx->anchor_valid = false;
     return KEYDIFF_OK;
 }
 
@@ -358,6 +390,7 @@ int keydiff_get_len(const keydiff_ctx* ctx, int32_t* len_out) {
 int keydiff_set_len(keydiff_ctx* ctx, int32_t len) {
     if (!ctx || len < 0 || len > ctx->cfg.budget) return KEYDIFF_ERR_INVALID_ARG;
     ctx->len = len;
+    ctx->anchor_valid = false;   // the caller brought its own cache contents
     return KEYDIFF_OK;
 }
 
