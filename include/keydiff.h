@@ -134,8 +134,26 @@ KEYDIFF_API int keydiff_evict_host(keydiff_ctx* ctx, void* k_cache, void* v_cach
 /* keydiff_destroy -- free the scratch and the ctx.  Synchronises the device.  NULL is OK. */
 KEYDIFF_API int keydiff_destroy(keydiff_ctx* ctx);
 
+/*
+ * keydiff_set_incremental -- choose how the fused path obtains the anchor of App. B.1 (first
+ * expression), mu = (1/n) sum_i k_i/||k_i||.  The cache is carried from block to block (Eq.
+ * block_processing), so the sum over a step's n rows is the sum over the rows already cached plus the
+ * sum over the B new rows.  With on != 0 (the default) the context keeps the cached rows' sum per unit
+ * on the device: an evicting step adds the block rows' terms, subtracts the evicted rows' terms (both
+ * recomputed from the same bf16 rows by the same arithmetic), and the next step needs only the block
+ * normalised before it can score.  The value is the same sum in a different order of additions (fp32
+ * partial sums folded in double precision); scores stay within the library's tolerance.  The running
+ * sum is rebuilt from all n rows on the first evicting step, after any append-only step,
+ * keydiff_set_len or keydiff_reset, and every 1024 evicting steps.  With on == 0 every step rebuilds it.
+ * REQUIREMENT with on != 0: between two keydiff_evict calls nobody else may change rows [0, len) of
+ * k_cache; after changing them call keydiff_set_len(ctx, len).  The staged path ignores the setting.
+ * Errors: INVALID_ARG (NULL ctx).
+ */
+KEYDIFF_API int keydiff_set_incremental(keydiff_ctx* ctx, int32_t on);
+
 /* Cache length bookkeeping (host side, no device work).  C_0 = empty: reset sets len = 0;
- * set_len resumes from a cache the caller restored (0 <= len <= N). */
+ * set_len resumes from a cache the caller restored (0 <= len <= N); both make the next evicting step
+ * rebuild the running anchor sum (keydiff_set_incremental). */
 KEYDIFF_API int keydiff_reset(keydiff_ctx* ctx);
 KEYDIFF_API int keydiff_get_len(const keydiff_ctx* ctx, int32_t* len_out);
 KEYDIFF_API int keydiff_set_len(keydiff_ctx* ctx, int32_t len);

@@ -24,7 +24,7 @@ KEYDIFF_PATH_AUTO, KEYDIFF_PATH_STAGED, KEYDIFF_PATH_FUSED = 0, 1, 2
 # every symbol include/keydiff.h declares
 EXPORTS = ["keydiff_create", "keydiff_evict", "keydiff_evict_host", "keydiff_destroy", "keydiff_reset",
            "keydiff_get_len", "keydiff_set_len", "keydiff_get_scratch", "keydiff_get_moved_rows",
-           "keydiff_get_launch_info", "keydiff_evict_static",
+           "keydiff_get_launch_info", "keydiff_evict_static", "keydiff_set_incremental",
            "keydiff_strerror", "keydiff_last_cuda_error"]
 
 
@@ -62,6 +62,7 @@ def load_library() -> ctypes.CDLL:
     lib.keydiff_reset.argtypes = [vp]
     lib.keydiff_get_len.argtypes = [vp, i32p]
     lib.keydiff_set_len.argtypes = [vp, i32]
+    lib.keydiff_set_incremental.argtypes = [vp, i32]
     lib.keydiff_get_scratch.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.keydiff_get_moved_rows.argtypes = [vp, ctypes.POINTER(vp)]
     lib.keydiff_get_launch_info.argtypes = [vp, i32p, i32p, i32p]
@@ -158,6 +159,10 @@ class KeyDiff:
 
     def reset(self):
         _check(self._lib.keydiff_reset(self._ctx))
+
+    def set_incremental(self, on: bool):
+        """``keydiff_set_incremental``: keep the anchor's running sum across steps (default) or rebuild it every step."""
+        _check(self._lib.keydiff_set_incremental(self._ctx, 1 if on else 0))
 
     def scratch(self):
         """Views (no copy) of the ctx-owned scratch: scores [U, N+max_block] fp32, kept_idx [U, N]

@@ -381,6 +381,12 @@ int keydiff_reset(keydiff_ctx* ctx) {
     return KEYDIFF_OK;
 }
 
+int keydiff_set_incremental(keydiff_ctx* ctx, int32_t on) {
+    if (!ctx) return KEYDIFF_ERR_INVALID_ARG;
+    ctx->incremental = on != 0;
+    return KEYDIFF_OK;
+}
+
 int keydiff_get_len(const keydiff_ctx* ctx, int32_t* len_out) {
     if (!ctx || !len_out) return KEYDIFF_ERR_INVALID_ARG;
     *len_out = ctx->len;

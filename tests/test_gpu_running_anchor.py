@@ -1,0 +1,93 @@
+"""GPU tests of the fused path's running anchor (the sum of k/||k|| over the cached rows kept across
+steps; App. B.1, first expression, split along Eq. block_processing): long streams against the oracle,
+agreement with the rebuild-every-step mode, invalidation by set_len, the periodic rebuild."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import compare
+from paper_2504_15364_b200 import KeyDiff, binding, synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def bits(t):
+    return t.detach().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def checked_step(kd, k_cache, v_cache, new_k, new_v):
+    N, length = kd.budget, kd.len
+    pre_k, pre_v = bits(k_cache), bits(v_cache)
+    kd.evict(k_cache, v_cache, new_k, new_v)
+    torch.cuda.synchronize()
+    sc = kd.scratch()
+    assert int(sc["status"].item()) == 0
+    return compare.check_step(pre_k, pre_v, length, bits(new_k), bits(new_v), N, bits(k_cache), bits(v_cache),
+                              sc["scores"].cpu().numpy(), sc["kept_idx"].cpu().numpy(), n_threads=8)
+
+
+def make(wl, incremental=True):
+    k_cache, v_cache, stream = synth.prefilled_cache(wl, DEV)
+    kd = KeyDiff(wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim, wl.budget, wl.block, path=binding.KEYDIFF_PATH_FUSED)
+    kd.set_incremental(incremental)
+    kd.set_len(wl.budget)
+    return kd, k_cache, v_cache, stream
+
+
+@pytest.mark.parametrize("model,N,B", [("outlier", 640, 64), ("drift", 1024, 32), ("clusters", 300, 7)])
+def test_long_stream_stays_inside_the_tolerance(model, N, B):
+    # 300 evicting steps on the running sum; the oracle checks the first steps, every 25th and the last
+    wl = synth.Workload("t", 1, 2, 3, 128, N, B, model, N + 300 * B, 21)
+    kd, k_cache, v_cache, stream = make(wl)
+    worst = 0.0
+    for step in range(300):
+        nk, nv = stream.next_block()
+        if step < 3 or step % 25 == 0 or step == 299:
+            worst = max(worst, checked_step(kd, k_cache, v_cache, nk, nv)["max_score_err_over_tol"])
+        else:
+            kd.evict(k_cache, v_cache, nk, nv)
+    assert worst < 0.5, f"score error reached {worst:.2f} of the tolerance"
+    kd.close()
+
+
+def test_agrees_with_rebuilding_every_step_and_is_deterministic():
+    wl = synth.Workload("t", 2, 1, 4, 128, 1536, 128, "outlier", 1536 + 40 * 128, 5)
+    runs = []
+    for incremental in (True, True, False):
+        kd, k_cache, v_cache, stream = make(wl, incremental)
+        for _ in range(40):
+            kd.evict(k_cache, v_cache, *stream.next_block())
+        torch.cuda.synchronize()
+        runs.append((k_cache.clone(), v_cache.clone(), kd.scratch()["scores"].clone()))
+        kd.close()
+    assert all(torch.equal(a, b) for a, b in zip(runs[0], runs[1])), "two runs on the running sum differ"
+    # against the rebuild mode: same cache unless a token sat inside the tolerance band of a threshold
+    same_rows = (runs[0][0] == runs[2][0]).all(dim=2).float().mean().item()
+    assert same_rows > 0.98
+    n = wl.budget + wl.block
+    assert torch.allclose(runs[0][2][:, :n], runs[2][2][:, :n], rtol=0, atol=2e-5) or same_rows < 1.0
+
+
+def test_set_len_after_outside_changes_rebuilds_the_sum():
+    wl = synth.Workload("t", 1, 1, 5, 128, 512, 64, "offset", 512 + 12 * 64, 8)
+    kd, k_cache, v_cache, stream = make(wl)
+    for _ in range(4):
+        checked_step(kd, k_cache, v_cache, *stream.next_block())
+    k_cache[:, 100:200] = k_cache[:, 100:200].flip(1) * 3      # the caller rewrites rows behind the library's back ...
+    kd.set_len(wl.budget)                                      # ... and says so
+    for _ in range(4):
+        checked_step(kd, k_cache, v_cache, *stream.next_block())
+    kd.close()
+
+
+def test_periodic_rebuild_after_1024_steps():
+    wl = synth.Workload("t", 1, 1, 2, 128, 96, 8, "offset", 96 + 1100 * 8, 13)
+    kd, k_cache, v_cache, stream = make(wl)
+    for step in range(1100):
+        nk, nv = stream.next_block()
+        if step in (0, 1, 1023, 1024, 1025, 1026, 1099):
+            checked_step(kd, k_cache, v_cache, nk, nv)
+        else:
+            kd.evict(k_cache, v_cache, nk, nv)
+    kd.close()
