@@ -225,6 +225,40 @@ __device__ __forceinline__ uint32_t row_score(const uint4& a, const uint4& b, co
     const float e = -(dot * approx_rcp(fmaxf(m * r, eps)));
     return order_key(e == 0.f ? 0.f : e);
 }
+// One lane's share of ||k||^2 and of mu.k (no exchange between lanes yet).
+__device__ __forceinline__ void lane_sumsq_dot(const uint4& a, const uint4& b, const float2 (&w)[8], float& ss, float& dot) {
+    float2 x[8];
+    unpack_pairs(a, b, x);
+    float2 s0 = make_float2(0.f, 0.f), s1 = s0, d0 = s0, d1 = s0;
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        s0 = __ffma2_rn(x[p], x[p], s0); s1 = __ffma2_rn(x[4 + p], x[4 + p], s1);
+        d0 = __ffma2_rn(x[p], w[p], d0); d1 = __ffma2_rn(x[4 + p], w[4 + p], d1);
+    }
+    ss = (s0.x + s0.y) + (s1.x + s1.y);
+    dot = (d0.x + d0.y) + (d1.x + d1.y);
+}
+// Eight values per lane, each to be summed over the 8 lanes of a row group: a butterfly that halves
+// the values it carries at every step (4 + 2 + 1 shuffles instead of 8 x 3).  Lane t (0..7 within the
+// group) returns the group's sum of v[t].
+__device__ __forceinline__ float group_sum8(const float (&v)[8], int t) {
+    float r4[4], r2[2];
+    const bool h4 = t & 4, h2 = t & 2, h1 = t & 1;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r4[i] = (h4 ? v[i + 4] : v[i]) + __shfl_xor_sync(0xffffffffu, h4 ? v[i] : v[i + 4], 4);
+#pragma unroll
+    for (int i = 0; i < 2; ++i) r2[i] = (h2 ? r4[i + 2] : r4[i]) + __shfl_xor_sync(0xffffffffu, h2 ? r4[i] : r4[i + 2], 2);
+    return (h1 ? r2[1] : r2[0]) + __shfl_xor_sync(0xffffffffu, h1 ? r2[0] : r2[1], 1);
+}
+// Keys of four rows of a row group from the lanes' shares v[2i] = ||k_i||^2, v[2i+1] = mu.k_i: after
+// the butterfly lane 2i holds row i's squared norm and fetches its dot product from lane 2i+1.
+// Returns row (t >> 1)'s key in the even lanes (odd lanes: unspecified).
+__device__ __forceinline__ uint32_t score4(const float (&v)[8], int t, float m, float eps) {
+    const float mine = group_sum8(v, t);
+    const float dot = __shfl_xor_sync(0xffffffffu, mine, 1);
+    const float e = -(dot * approx_rcp(fmaxf(m * approx_sqrt(mine), eps)));
+    return order_key(e == 0.f ? 0.f : e);
+}
 // Step a2 for one row: orderable key of e = -(mu.k)/max(||mu|| ||k||, eps), -0 mapped to +0.
 __device__ __forceinline__ uint32_t row_a2(const uint4& a, const uint4& b, const float2 (&w)[8], float m, float r, float eps) {
     float2 x[8];
@@ -532,28 +566,29 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 if (tile >= ntiles) break;
                 mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
                 parity ^= 1u << s;
-#pragma unroll 1
-                for (int half = 0; half < 2; ++half) {
-                    uint4 a[2], b[2];
+                float v[8];   // this lane's shares of the tile's four rows of its row group
 #pragma unroll
-                    for (int it = 0; it < 2; ++it) {
-                        const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
-                        a[it] = make_uint4(0, 0, 0, 0); b[it] = a[it];
-                        if (lr < rs) { a[it] = rows[lr * kRowVec + t]; b[it] = rows[lr * kRowVec + t + 8]; }
-                    }
-#pragma unroll
-                    for (int it = 0; it < 2; ++it) {
-                        const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
-                        const uint32_t key = row_score(a[it], b[it], w, m, p.eps);
-                        if (lr < rs && t == 0) keys[seg_a + lr] = key;
-                    }
+                for (int it = 0; it < 4; ++it) {
+                    const int lr = tile * kTileRows + it * 4 + sub;
+                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
+                    if (lr < rs) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
+                    lane_sumsq_dot(a, b, w, v[2 * it], v[2 * it + 1]);
                 }
+                const uint32_t key = score4(v, t, m, p.eps);
+                const int lr = tile * kTileRows + (t >> 1) * 4 + sub;
+                if (!(t & 1) && lr < rs) keys[seg_a + lr] = key;
             }
 #pragma unroll
-            for (int k = 0; k < kRegRows; ++k) {
-                const uint32_t key = row_score(ra[k], rb[k], w, m, p.eps);
-                const int lr = rs + k * kGroups + g;
-                if (lr < seg && t == 0) keys[seg_a + lr] = key;
+            for (int k0 = 0; k0 < kRegRows; k0 += 4) {   // register rows, four at a time
+                float v[8];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (k0 + i < kRegRows) lane_sumsq_dot(ra[k0 + i], rb[k0 + i], w, v[2 * i], v[2 * i + 1]);
+                    else { v[2 * i] = 0.f; v[2 * i + 1] = 0.f; }
+                }
+                const uint32_t key = score4(v, t, m, p.eps);
+                const int lr = rs + (k0 + (t >> 1)) * kGroups + g;
+                if (!(t & 1) && k0 + (t >> 1) < kRegRows && lr < seg) keys[seg_a + lr] = key;
             }
         }
         } else {
