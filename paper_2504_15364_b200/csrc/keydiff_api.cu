@@ -177,14 +177,16 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     p.anchor_out = c->anchor_sum[c->anchor_par ^ 1];
     p.anchor_delta = c->anchor_delta;
     const int nclusters = std::min(c->U, c->fused_max_clusters);
-    // Start-up stagger: one unit's estimated duration spread evenly over the co-resident clusters.
-    // A unit moves 4 slices (K in, K out, V in, V out) per SM at roughly 45 GB/s per SM when the other
-    // SMs are busy too, plus a few microseconds of arithmetic and barriers.
+    // Start-up stagger: somewhat less than one unit's duration spread evenly over the co-resident
+    // clusters.  A unit moves 4 slices (K in, K out, V in, V out) per SM at roughly 60 GB/s per SM when
+    // the other SMs are busy too, plus a few microseconds of arithmetic and barriers (a sweep of the
+    // delay on a B200 put the best value at 0.7-0.95 of unit time / clusters for the large workloads).
     p.stagger_ns = 0;
     if (nclusters > 1 && c->U > nclusters) {
-        const double unit_ns = 4.0 * p.rows_per_cta * kRowBytes / 45.0 + 8000.0;
+        const double unit_ns = 4.0 * p.rows_per_cta * kRowBytes / 60.0 + 6000.0;
         p.stagger_ns = static_cast<unsigned>(unit_ns / nclusters);
     }
+    if (const char* env = std::getenv("KEYDIFF_STAGGER_NS")) p.stagger_ns = static_cast<unsigned>(std::atoi(env));   // tuning aid
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(nclusters * c->cluster);
     cfg.blockDim = dim3(kFusedThreads);
