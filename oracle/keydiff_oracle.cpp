@@ -32,6 +32,16 @@
 //     scores the older token is kept;
 //   - kept rows are written in original token order (ascending index).
 //
+// Two variants of the method are restated as well (the *_ex entry points):
+//   * raw-mean anchor (anchor_mode 1) -- Sec. 3.2, the sentence after Eq. (efficient-keydiff) and
+//     the caption of the method figure: the anchor is the mean of the keys themselves,
+//     mu(K) = (1/n) sum_i k_i; the score formula is unchanged.
+//   * sliding window (recent_window w) -- Sec. 3.2, "KeyDiff with sliding window": part of the
+//     budget is reserved for the most recent tokens and KeyDiff manages the rest.  Reading (the
+//     paper gives no formula): the last w of the n tokens are always kept, the N - w tokens with
+//     the largest eviction score are kept among the first n - w, and the anchor is still formed
+//     from all n keys.
+//
 // Every function is pinned by tests that do not call back into this file:
 // hand-worked examples, closed forms, the pairwise identity evaluated in numpy,
 // brute force over all subsets, and structural invariants.  No function here is
@@ -61,8 +71,9 @@ inline double bf16_bits_to_double(uint16_t bits) {
 // App. B.1, both expressions.  K is n x d row-major doubles.
 // Outputs (any may be null): r[n] key norms, mu[d] anchor, *m anchor norm,
 // s[n] cosine similarities of each key to the anchor.
+// anchor_mode 0: mu = mean of k_i/||k_i|| (the equation); 1: mu = mean of k_i (Sec. 3.2, text).
 void scores_f64(const double* K, int64_t n, int64_t d, double eps,
-                double* r_out, double* mu_out, double* m_out, double* s_out) {
+                double* r_out, double* mu_out, double* m_out, double* s_out, int anchor_mode = 0) {
     std::vector<double> r(n), mu(d, 0.0);
     // ||k_i|| = sqrt(k_i . k_i)
     for (int64_t i = 0; i < n; ++i) {
@@ -72,7 +83,7 @@ void scores_f64(const double* K, int64_t n, int64_t d, double eps,
     }
     // mu = (1/n) sum_i k_i / ||k_i||   (guarded divisor, see header)
     for (int64_t i = 0; i < n; ++i) {
-        const double div = std::max(r[i], eps);
+        const double div = anchor_mode == 1 ? 1.0 : std::max(r[i], eps);   // raw mean: mu = (1/n) sum_i k_i
         for (int64_t c = 0; c < d; ++c) mu[c] += K[i * d + c] / div;
     }
     for (int64_t c = 0; c < d; ++c) mu[c] /= static_cast<double>(n);
@@ -115,12 +126,28 @@ int64_t select_topn(const double* e, int64_t n, int64_t N, int64_t* S_out,
     return keep;
 }
 
+// Sliding window: the last w of the n tokens are kept unconditionally; among the first n - w the
+// N - w with the largest e are kept (same order and tie rule).  Requires 0 <= w <= N.  tau = score of
+// the last token kept by the score rule (0 if none is).
+int64_t select_topn_window(const double* e, int64_t n, int64_t N, int64_t w, int64_t* S_out, double* tau_out) {
+    if (n <= N) return select_topn(e, n, N, S_out, tau_out);
+    const int64_t head = n - w;                       // tokens the score rule decides on
+    std::vector<int64_t> S(N);
+    double tau = 0.0;
+    const int64_t kept_head = head > 0 ? select_topn(e, head, N - w, S.data(), &tau) : 0;   // == N - w
+    for (int64_t j = 0; j < w; ++j) S[kept_head + j] = head + j;                            // the window, in order
+    std::copy(S.begin(), S.begin() + kept_head + w, S_out);
+    if (tau_out) *tau_out = tau;
+    return kept_head + w;
+}
+
 struct HeadArgs {
     const uint16_t* k_cache; const uint16_t* v_cache; int64_t len;
     const uint16_t* new_k;   const uint16_t* new_v;   int64_t B;
     int64_t N; int64_t d; double eps;
     uint16_t* k_out; uint16_t* v_out; int64_t* len_out;
     double* e_out; int64_t* S_out; double* tau_out; double* m_out;
+    int anchor_mode = 0; int64_t window = 0;
 };
 
 // One unit (one KV head of one layer of one sequence), Eq. (eviction_policy)
@@ -139,9 +166,9 @@ void evict_head(const HeadArgs& a) {
         std::vector<double> K(static_cast<size_t>(n) * d), s(n), e(n);
         for (int64_t i = 0; i < n; ++i)
             for (int64_t c = 0; c < d; ++c) K[i * d + c] = bf16_bits_to_double(k_row(i)[c]);
-        scores_f64(K.data(), n, d, a.eps, nullptr, nullptr, &m, s.data());
+        scores_f64(K.data(), n, d, a.eps, nullptr, nullptr, &m, s.data(), a.anchor_mode);
         for (int64_t i = 0; i < n; ++i) e[i] = eviction_score(s[i]);
-        select_topn(e.data(), n, a.N, S.data(), &tau);
+        select_topn_window(e.data(), n, a.N, a.window, S.data(), &tau);
         if (a.e_out) std::copy(e.begin(), e.end(), a.e_out);
     }
     // gather(K,S), gather(V,S): bit-exact row copies in token order
@@ -163,6 +190,17 @@ extern "C" {
 void kd_oracle_scores(const double* K, int64_t n, int64_t d, double eps,
                       double* r, double* mu, double* m, double* s) {
     scores_f64(K, n, d, eps, r, mu, m, s);
+}
+
+// The same with the anchor variant chosen: 0 = mean of normalised keys, 1 = mean of raw keys.
+void kd_oracle_scores_ex(const double* K, int64_t n, int64_t d, double eps, int32_t anchor_mode,
+                         double* r, double* mu, double* m, double* s) {
+    scores_f64(K, n, d, eps, r, mu, m, s, anchor_mode);
+}
+
+// Kept indices (ascending) with a window of w always-kept most recent tokens; returns the count.
+int64_t kd_oracle_select_window(const double* e, int64_t n, int64_t N, int64_t w, int64_t* S, double* tau) {
+    return select_topn_window(e, n, N, w, S, tau);
 }
 
 // e[i] = eviction score of cosine s[i].
@@ -238,6 +276,25 @@ int32_t kd_oracle_evict_units_bf16(const uint16_t* k_cache, const uint16_t* v_ca
         pool.emplace_back([&, t] { for (int64_t u = t; u < U; u += T) run_unit(u); });
     for (auto& th : pool) th.join();
     return T;
+}
+
+// The same with the anchor variant and the sliding window chosen (single-threaded per call; the
+// Python wrapper spreads units over threads by calling it on slices).
+void kd_oracle_evict_units_bf16_ex(const uint16_t* k_cache, const uint16_t* v_cache, int64_t len,
+                                   const uint16_t* new_k, const uint16_t* new_v, int64_t B,
+                                   int64_t N, int64_t d, double eps, int64_t U, int32_t anchor_mode, int64_t window,
+                                   uint16_t* k_out, uint16_t* v_out,
+                                   double* e_out, int64_t* S_out, double* tau_out, double* m_out) {
+    const int64_t n = len + B;
+    for (int64_t u = 0; u < U; ++u) {
+        HeadArgs a{k_cache + u * N * d, v_cache + u * N * d, len, new_k + u * B * d, new_v + u * B * d, B, N, d, eps,
+                   k_out + u * N * d, v_out + u * N * d, nullptr,
+                   e_out ? e_out + u * n : nullptr, S_out ? S_out + u * N : nullptr,
+                   tau_out ? tau_out + u : nullptr, m_out ? m_out + u : nullptr};
+        a.anchor_mode = anchor_mode;
+        a.window = window;
+        evict_head(a);
+    }
 }
 
 }  // extern "C"

@@ -56,6 +56,13 @@ def _load():
         lib.kd_oracle_evict_units_bf16.argtypes = [c_hp, c_hp, i64, c_hp, c_hp, i64, i64, i64, f64, i64,
                                                    c_hp, c_hp, c_dp, c_ip, c_dp, c_dp, ctypes.c_int32]
         lib.kd_oracle_evict_units_bf16.restype = ctypes.c_int32
+        lib.kd_oracle_scores_ex.argtypes = [c_dp, i64, i64, f64, ctypes.c_int32, c_dp, c_dp, c_dp, c_dp]
+        lib.kd_oracle_scores_ex.restype = None
+        lib.kd_oracle_select_window.argtypes = [c_dp, i64, i64, i64, c_ip, c_dp]
+        lib.kd_oracle_select_window.restype = i64
+        lib.kd_oracle_evict_units_bf16_ex.argtypes = [c_hp, c_hp, i64, c_hp, c_hp, i64, i64, i64, f64, i64,
+                                                      ctypes.c_int32, i64, c_hp, c_hp, c_dp, c_ip, c_dp, c_dp]
+        lib.kd_oracle_evict_units_bf16_ex.restype = None
         _lib = lib
     return _lib
 
@@ -72,13 +79,14 @@ def _hp(a):
     return a.ctypes.data_as(ctypes.POINTER(ctypes.c_uint16))
 
 
-def scores(K, eps: float = DEFAULT_EPS):
-    """K: (n, d) float64.  Returns dict r (n,), mu (d,), m (float), s (n,) cosines."""
+def scores(K, eps: float = DEFAULT_EPS, anchor_mode: int = 0):
+    """K: (n, d) float64.  Returns dict r (n,), mu (d,), m (float), s (n,) cosines.
+    anchor_mode 0: anchor = mean of normalised keys; 1: mean of the raw keys."""
     K = np.ascontiguousarray(K, dtype=np.float64)
     n, d = K.shape
     r, mu, s = np.empty(n), np.empty(d), np.empty(n)
     m = np.empty(1)
-    _load().kd_oracle_scores(_dp(K), n, d, eps, _dp(r), _dp(mu), _dp(m), _dp(s))
+    _load().kd_oracle_scores_ex(_dp(K), n, d, eps, anchor_mode, _dp(r), _dp(mu), _dp(m), _dp(s))
     return {"r": r, "mu": mu, "m": float(m[0]), "s": s}
 
 
@@ -89,13 +97,14 @@ def eviction_scores(s):
     return e
 
 
-def select(e, N: int):
-    """Kept token indices (ascending) and the threshold tau (N-th largest e)."""
+def select(e, N: int, recent_window: int = 0):
+    """Kept token indices (ascending) and the threshold tau (score of the last token the score rule
+    keeps).  recent_window w: the last w tokens are always kept, the rest compete for N - w places."""
     e = np.ascontiguousarray(e, dtype=np.float64)
     keep = min(N, e.size)
     S = np.empty(keep, dtype=np.int64)
     tau = np.empty(1)
-    got = _load().kd_oracle_select(_dp(e), e.size, N, _ip(S), _dp(tau))
+    got = _load().kd_oracle_select_window(_dp(e), e.size, N, recent_window, _ip(S), _dp(tau))
     assert got == keep
     return S, float(tau[0])
 
@@ -109,7 +118,7 @@ def pairwise_rowsum(K):
 
 
 def evict_units_bf16(k_cache, v_cache, length: int, new_k, new_v, N: int,
-                     eps: float = DEFAULT_EPS, n_threads: int = 1):
+                     eps: float = DEFAULT_EPS, n_threads: int = 1, anchor_mode: int = 0, recent_window: int = 0):
     """U independent units on bf16 bit patterns (uint16 arrays).
 
     k_cache, v_cache: (U, N, d) uint16 with rows [0, length) valid; new_k, new_v:
@@ -133,8 +142,23 @@ def evict_units_bf16(k_cache, v_cache, length: int, new_k, new_v, N: int,
     e = np.zeros((U, n), dtype=np.float64)
     S_full = np.zeros((U, N), dtype=np.int64)
     tau, m = np.zeros(U), np.zeros(U)
-    used = _load().kd_oracle_evict_units_bf16(
-        _hp(k_cache), _hp(v_cache), length, _hp(new_k), _hp(new_v), B, N, d, eps, U,
-        _hp(k_out), _hp(v_out), _dp(e), _ip(S_full), _dp(tau), _dp(m), n_threads)
+    if anchor_mode == 0 and recent_window == 0:
+        used = _load().kd_oracle_evict_units_bf16(
+            _hp(k_cache), _hp(v_cache), length, _hp(new_k), _hp(new_v), B, N, d, eps, U,
+            _hp(k_out), _hp(v_out), _dp(e), _ip(S_full), _dp(tau), _dp(m), n_threads)
+    else:
+        assert 0 <= recent_window <= N
+        from concurrent.futures import ThreadPoolExecutor
+        used = max(1, min(n_threads, U))
+        lib = _load()
+
+        def run(t):   # units t, t+used, ...: one C call per unit (ctypes drops the GIL)
+            for u in range(t, U, used):
+                lib.kd_oracle_evict_units_bf16_ex(
+                    _hp(k_cache[u]), _hp(v_cache[u]), length, _hp(new_k[u]), _hp(new_v[u]), B, N, d, eps, 1,
+                    anchor_mode, recent_window, _hp(k_out[u]), _hp(v_out[u]), _dp(e[u]), _ip(S_full[u]),
+                    _dp(tau[u:u + 1]), _dp(m[u:u + 1]))
+        with ThreadPoolExecutor(used) as pool:
+            list(pool.map(run, range(used)))
     return {"k": k_out, "v": v_out, "len": keep, "e": e if n > N else None,
             "S": S_full[:, :keep].copy(), "tau": tau, "m": m, "threads": int(used)}
