@@ -61,6 +61,14 @@ enum {
 
 enum { KEYDIFF_BF16 = 0 };
 
+/* The anchor of Eq. (efficient-keydiff).  The equation and App. B.1 use the mean of the normalised
+ * keys; the text that follows the equation says the mean of the keys themselves serves as well.  Both
+ * are built; the score formula s_i = mu.k_i / max(||mu|| ||k_i||, eps) is the same. */
+enum {
+    KEYDIFF_ANCHOR_NORMALISED = 0,  /* mu = (1/n) sum_i k_i/||k_i||   (default) */
+    KEYDIFF_ANCHOR_RAW_MEAN = 1     /* mu = (1/n) sum_i k_i */
+};
+
 /* Which kernels serve keydiff_evict. */
 enum {
     KEYDIFF_PATH_AUTO = 0,    /* fused cluster kernel when a unit fits, else the staged kernels */
@@ -80,6 +88,9 @@ typedef struct {
     int32_t path;          /* KEYDIFF_PATH_* */
     float   eps;           /* eps of App. B.1's max(.,eps); 0 selects the default 1e-8 */
     int32_t device;        /* CUDA device ordinal */
+    int32_t anchor_mode;   /* KEYDIFF_ANCHOR_*: which mean is the anchor (Sec. 3.2) */
+    int32_t recent_window; /* w >= 0 most recent tokens that are never evicted (Sec. 3.2, "KeyDiff with
+                              sliding window"); 0 = plain KeyDiff; w <= budget */
 } keydiff_config;
 
 /*
@@ -87,7 +98,8 @@ typedef struct {
  * n_kv_heads units (scores U*(N+max_block) fp32, kept-index list U*N int32, anchor
  * partials, per-unit counters, one status word).  Synchronous.  *out is set only on
  * KEYDIFF_OK.  The initial cache length is 0 (C_0 = empty, Eq. block_processing).
- * Errors: INVALID_ARG (NULL, non-positive sizes), UNSUPPORTED (dtype, head_dim, a unit
+ * Errors: INVALID_ARG (NULL, non-positive sizes, unknown anchor_mode, recent_window outside
+ * [0, budget]), UNSUPPORTED (dtype, head_dim, a unit
  * too large for the requested path, no sm_100 device), ALLOC, CUDA.
  */
 KEYDIFF_API int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out);
@@ -102,6 +114,9 @@ KEYDIFF_API int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out);
  *   kept (ties: lower token index wins), and K and V are compacted in place in
  *   original token order; rows in front of the first evicted row are not touched.
  *   Afterwards len = min(N, n) for every unit.
+ *   With recent_window = w > 0 (Sec. 3.2, sliding window; the paper gives no formula, this is the
+ *   reading taken): the last w of the n tokens are always kept, the N - w tokens with the largest e are
+ *   kept among the first n - w, and the anchor is still formed from all n keys.
  * k_cache, v_cache: device, in/out, caller-owned.  new_k, new_v: device, read only,
  * caller-owned; they may be reused once the work enqueued on `stream` has completed.
  * budget_N, n_kv_heads, head_dim restate the ctx's values and must equal them;

@@ -29,16 +29,19 @@ def _bf16_to_f64(bits: np.ndarray) -> np.ndarray:
 
 
 def check_step(k_cache, v_cache, length, new_k, new_v, N, gpu_k, gpu_v, gpu_scores, gpu_kept,
-               eps=oracle.DEFAULT_EPS, units=None, n_threads=1):
+               eps=oracle.DEFAULT_EPS, units=None, n_threads=1, anchor_mode=0, recent_window=0):
     """All array arguments are host numpy arrays: uint16 bit patterns [U, rows, d] for K/V,
     float32 [U, >=n] for gpu_scores, int32 [U, N] for gpu_kept.  ``units`` restricts the check to
-    a subset of unit indices.  Returns a report dict; raises AssertionError on a violation."""
+    a subset of unit indices.  anchor_mode / recent_window select the method's variants (raw-mean anchor;
+    the last recent_window tokens always kept).  Returns a report dict; raises AssertionError on a violation."""
     U = k_cache.shape[0]
     sel = np.arange(U) if units is None else np.asarray(units)
     B = new_k.shape[1]
     n = length + B
     assert n > N, "check_step is for evicting steps"
-    ref = oracle.evict_units_bf16(k_cache[sel], v_cache[sel], length, new_k[sel], new_v[sel], N, eps, n_threads)
+    ref = oracle.evict_units_bf16(k_cache[sel], v_cache[sel], length, new_k[sel], new_v[sel], N, eps, n_threads,
+                                  anchor_mode=anchor_mode, recent_window=recent_window)
+    w = recent_window
     rep = {"units": len(sel), "n": n, "max_score_err_over_tol": 0.0, "max_plain_rel": 0.0,
            "set_mismatch_in_band": 0, "min_anchor_norm": float(ref["m"].min())}
     for j, u in enumerate(sel):
@@ -51,7 +54,7 @@ def check_step(k_cache, v_cache, length, new_k, new_v, N, gpu_k, gpu_v, gpu_scor
         if ref["m"][j] >= MIN_ANCHOR_NORM:
             K = _bf16_to_f64(allk)
             r = np.sqrt((K * K).sum(1))
-            unit = K / np.maximum(r, eps)[:, None]
+            unit = K if anchor_mode == 1 else K / np.maximum(r, eps)[:, None]
             mu = unit.sum(0) / n
             kappa = (np.abs(K) @ np.abs(mu)) / np.maximum(np.sqrt((mu * mu).sum()) * r, eps)
             tol = SCORE_RTOL * np.maximum(np.abs(e_ref), kappa)
@@ -69,8 +72,9 @@ def check_step(k_cache, v_cache, length, new_k, new_v, N, gpu_k, gpu_v, gpu_scor
         assert len(S_gpu) == N and (np.diff(S_gpu) > 0).all() and S_gpu[0] >= 0 and S_gpu[-1] < n, \
             f"unit {u}: kept list is not N ascending in-range indices"
         e32 = gpu_scores[u, :n]
-        order = np.lexsort((np.arange(n), -e32.astype(np.float64)))     # e desc, index asc
-        want = np.sort(order[:N])
+        head = n - w                                                     # tokens the score rule decides on
+        order = np.lexsort((np.arange(head), -e32[:head].astype(np.float64)))     # e desc, index asc
+        want = np.sort(np.concatenate([order[:N - w], np.arange(head, n)]))
         assert (S_gpu == want).all(), f"unit {u}: kept set is not the top-N of the GPU's own scores"
         # ---- selection: agreement with the oracle outside the threshold band
         S_ref = ref["S"][j]

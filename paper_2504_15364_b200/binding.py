@@ -20,6 +20,7 @@ KEYDIFF_ERR_CUDA, KEYDIFF_ERR_STATE, KEYDIFF_ERR_TIMEOUT = -4, -5, -6
 KEYDIFF_ERR_TOO_LARGE = -7
 KEYDIFF_BF16 = 0
 KEYDIFF_PATH_AUTO, KEYDIFF_PATH_STAGED, KEYDIFF_PATH_FUSED = 0, 1, 2
+KEYDIFF_ANCHOR_NORMALISED, KEYDIFF_ANCHOR_RAW_MEAN = 0, 1
 
 # every symbol include/keydiff.h declares
 EXPORTS = ["keydiff_create", "keydiff_evict", "keydiff_evict_host", "keydiff_destroy", "keydiff_reset",
@@ -32,7 +33,7 @@ class keydiff_config(ctypes.Structure):
     _fields_ = [("n_layers", ctypes.c_int32), ("batch", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("budget", ctypes.c_int32), ("max_block", ctypes.c_int32),
                 ("dtype", ctypes.c_int32), ("path", ctypes.c_int32), ("eps", ctypes.c_float),
-                ("device", ctypes.c_int32)]
+                ("device", ctypes.c_int32), ("anchor_mode", ctypes.c_int32), ("recent_window", ctypes.c_int32)]
 
 
 class KeyDiffError(RuntimeError):
@@ -99,13 +100,14 @@ class KeyDiff:
     """
 
     def __init__(self, n_layers: int, batch: int, n_kv_heads: int, head_dim: int, budget: int, max_block: int,
-                 *, path: int = KEYDIFF_PATH_AUTO, eps: float = 0.0, device: int | None = None):
+                 *, path: int = KEYDIFF_PATH_AUTO, eps: float = 0.0, device: int | None = None,
+                 anchor_mode: int = KEYDIFF_ANCHOR_NORMALISED, recent_window: int = 0):
         self._lib = load_library()
         self._ctx = ctypes.c_void_p()
         if device is None:
             device = torch.cuda.current_device() if torch.cuda.is_available() else 0
         self.cfg = keydiff_config(n_layers, batch, n_kv_heads, head_dim, budget, max_block, KEYDIFF_BF16, path,
-                                  eps, device)
+                                  eps, device, anchor_mode, recent_window)
         _check(self._lib.keydiff_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx)))
         self.units = n_layers * batch * n_kv_heads
         self.budget, self.max_block, self.head_dim, self.n_kv_heads = budget, max_block, head_dim, n_kv_heads

@@ -94,6 +94,8 @@ struct FusedParams {
     // = anchor_in[u][c] + sum over CTA ranks r of anchor_delta[u][r][c]; this step writes anchor_out and
     // new deltas
     const double* anchor_in; double* anchor_out; float* anchor_delta;
+    int raw_anchor;     // 1: the anchor is the mean of the keys themselves (Sec. 3.2), 0: of the normalised keys
+    int window;         // w most recent tokens that are never evicted (Sec. 3.2, sliding window)
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -206,11 +208,12 @@ __device__ __forceinline__ float pairs_dot(const float2 (&x)[8], const float2 (&
 // Step a1 for one row: returns ||k||; adds k / max(||k||, eps) into acc when the row is valid.
 // 1/max(r, eps) = min(1/r, 1/eps); the reciprocal square root and the square root are the
 // hardware approximations (relative error about 2^-22, far inside the score tolerance).
-__device__ __forceinline__ float row_a1(const uint4& a, const uint4& b, bool valid, float inv_eps, float2 (&acc)[8]) {
+// raw: the anchor is the mean of the keys themselves (Sec. 3.2), so k is added as it is.
+__device__ __forceinline__ float row_a1(const uint4& a, const uint4& b, bool valid, float inv_eps, float2 (&acc)[8], bool raw) {
     float2 x[8];
     unpack_pairs(a, b, x);
     const float ss = pairs_sumsq(x);
-    const float inv = valid ? fminf(approx_rsqrt(ss), inv_eps) : 0.f;
+    const float inv = valid ? (raw ? 1.0f : fminf(approx_rsqrt(ss), inv_eps)) : 0.f;
     const float2 inv2 = make_float2(inv, inv);
 #pragma unroll
     for (int p = 0; p < 8; ++p) acc[p] = __ffma2_rn(x[p], inv2, acc[p]);
@@ -442,6 +445,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     const int cluster_id = blockIdx.x / C, nclusters = gridDim.x / C;
     const int len = p.len, B = p.B, N = p.N, n = len + B, E = n - N;   // E tokens are evicted
     const float inv_eps = 1.0f / p.eps;
+    const bool raw = p.raw_anchor != 0;
     // fast select: evicted-token bitmap, its per-word prefix and the threshold bin's keys share `xchg`
     const int nwords = (n + 31) >> 5;
     uint32_t* bitmap = reinterpret_cast<uint32_t*>(smem + L.xchg);
@@ -521,7 +525,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                     const uint4* row = p.new_k + (static_cast<size_t>(u) * B + br) * kRowVec;
                     a = row[t]; b = row[t + 8];
                 }
-                row_a1(a, b, br < B, inv_eps, acc);
+                row_a1(a, b, br < B, inv_eps, acc, raw);
             }
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
@@ -614,13 +618,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
 #pragma unroll
                 for (int it = 0; it < 2; ++it) {
                     const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
-                    const float r = row_a1(a[it], b[it], lr < rs, inv_eps, acc);
+                    const float r = row_a1(a[it], b[it], lr < rs, inv_eps, acc, raw);
                     if (lr < rs && t == 0) keys[seg_a + lr] = __float_as_uint(r);   // parked in the row's key slot until a2
                 }
             }
         }
 #pragma unroll
-        for (int k = 0; k < kRegRows; ++k) rn[k] = row_a1(ra[k], rb[k], rs + k * kGroups + g < seg, inv_eps, acc);
+        for (int k = 0; k < kRegRows; ++k) rn[k] = row_a1(ra[k], rb[k], rs + k * kGroups + g < seg, inv_eps, acc, raw);
         // CTA reduction: 4 groups of a warp by shuffle, 16 warps through shared memory, fixed order
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -714,6 +718,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             }
         }
         cluster_wait();       // (2) the key table of every CTA holds all n keys
+        if (p.window > 0) {
+            // sliding window (Sec. 3.2): the last `window` tokens get the largest possible key, so they are
+            // never among the E smallest; the scores in global scratch stay what they are
+            __syncthreads();   // this CTA's score write-out has read its keys
+            for (int i = n - p.window + tid; i < n; i += kFusedThreads) keys[i] = 0xffffffffu;
+            __syncthreads();
+        }
         // ------------------------------------------------------------ a3 + plan: who is evicted, where every kept row goes
         bool planned = false;
         if (fast_ok) {
@@ -857,7 +868,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 const bool vis = lr < seg && lr >= skip_local;
                 const int d = vis ? dst_of[lr] : 0;
                 if (vis && d >= 0) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
-                if (__any_sync(0xffffffffu, vis && d < 0)) row_a1(ra[k], rb[k], vis && d < 0, inv_eps, gone);
+                if (__any_sync(0xffffffffu, vis && d < 0)) row_a1(ra[k], rb[k], vis && d < 0, inv_eps, gone, raw);
                 if (vis) {
                     const uint4* row = concat_row(p.v_cache, p.new_v, u, seg_a + lr, len, B, N);
                     ra[k] = row[t]; rb[k] = row[t + 8];
@@ -876,7 +887,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                     uint4 a = make_uint4(0, 0, 0, 0), b = a;
                     if (vis) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
                     if (vis && d >= 0) { out[d * kRowVec + t] = a; out[d * kRowVec + t + 8] = b; }
-                    if (__any_sync(0xffffffffu, vis && d < 0)) row_a1(a, b, vis && d < 0, inv_eps, gone);
+                    if (__any_sync(0xffffffffu, vis && d < 0)) row_a1(a, b, vis && d < 0, inv_eps, gone, raw);
                 }
                 // The tile's only readers are this warp's lanes and their reads have returned (the stores
                 // above consumed them), so the copy engine may overwrite it: a write after reads needs

@@ -176,6 +176,8 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     p.anchor_in = c->anchor_sum[c->anchor_par];
     p.anchor_out = c->anchor_sum[c->anchor_par ^ 1];
     p.anchor_delta = c->anchor_delta;
+    p.raw_anchor = c->cfg.anchor_mode == KEYDIFF_ANCHOR_RAW_MEAN;
+    p.window = c->cfg.recent_window;
     const int nclusters = std::min(c->U, c->fused_max_clusters);
     // Start-up stagger: somewhat less than one unit's duration spread evenly over the co-resident
     // clusters.  A unit moves 4 slices (K in, K out, V in, V out) per SM at roughly 60 GB/s per SM when
@@ -210,11 +212,11 @@ int launch_staged(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const u
     const int rows_per_split = (n + c->splits - 1) / c->splits;
     const dim3 grid(c->splits, U);
     anchor_partial_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, c->len, B, N, c->eps, rows_per_split, c->nmax,
-                                                           c->partial, c->norms);
+                                                           c->partial, c->norms, c->cfg.anchor_mode == KEYDIFF_ANCHOR_RAW_MEAN);
     score_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, c->len, B, N, c->eps, rows_per_split, c->nmax,
                                                   c->partial, c->norms, c->scores);
     select_kernel<<<U, kSelectThreads, static_cast<size_t>(n) * 4, st>>>(c->scores, n, N, c->nmax, c->len, c->kept_idx,
-                                                                          c->first_evicted, c->moved_rows);
+                                                                          c->first_evicted, c->moved_rows, c->cfg.recent_window);
     compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, c->len, B, N, c->kept_idx, c->first_evicted);
     KD_CUDA(cudaGetLastError());
     return KEYDIFF_OK;
@@ -231,6 +233,8 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
         return KEYDIFF_ERR_INVALID_ARG;
     if (cfg->path != KEYDIFF_PATH_AUTO && cfg->path != KEYDIFF_PATH_STAGED && cfg->path != KEYDIFF_PATH_FUSED)
         return KEYDIFF_ERR_INVALID_ARG;
+    if (cfg->anchor_mode != KEYDIFF_ANCHOR_NORMALISED && cfg->anchor_mode != KEYDIFF_ANCHOR_RAW_MEAN) return KEYDIFF_ERR_INVALID_ARG;
+    if (cfg->recent_window < 0 || cfg->recent_window > cfg->budget) return KEYDIFF_ERR_INVALID_ARG;
     if (cfg->dtype != KEYDIFF_BF16 || cfg->head_dim != kd::kHeadDim) return KEYDIFF_ERR_UNSUPPORTED;
     const long long U = 1LL * cfg->n_layers * cfg->batch * cfg->n_kv_heads;
     const long long nmax = 1LL * cfg->budget + cfg->max_block;
@@ -542,9 +546,9 @@ extern "C" int keydiff_evict_static(void* k_cache, void* v_cache, const void* ne
     const int nn = static_cast<int>(n);
     const int rows_per_split = (nn + splits - 1) / splits;
     const dim3 grid(splits, U);
-    anchor_partial_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, len, block_B, N, e, rows_per_split, nn, partial, norms);
+    anchor_partial_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, len, block_B, N, e, rows_per_split, nn, partial, norms, 0);
     score_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, len, block_B, N, e, rows_per_split, nn, partial, norms, scores);
-    select_kernel<<<U, kSelectThreads, static_cast<size_t>(nn) * 4, st>>>(scores, nn, N, nn, len, kept, first, moved);
+    select_kernel<<<U, kSelectThreads, static_cast<size_t>(nn) * 4, st>>>(scores, nn, N, nn, len, kept, first, moved, 0);
     compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, len, block_B, N, kept, first);
     KD_CUDA(cudaGetLastError());
     return KEYDIFF_OK;

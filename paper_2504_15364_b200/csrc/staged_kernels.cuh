@@ -20,11 +20,11 @@ __device__ __forceinline__ const uint4* concat_row(const uint4* cache, const uin
 }
 
 // Step a1 (App. B.1, first expression): per key ||k_i|| and the partial sum of k_i/max(||k_i||,eps)
-// over this CTA's slice of rows.  grid = (splits, U).
+// (of k_i itself for the raw-mean anchor of Sec. 3.2) over this CTA's slice of rows.  grid = (splits, U).
 __global__ void __launch_bounds__(kStagedThreads)
 anchor_partial_kernel(const uint4* __restrict__ k_cache, const uint4* __restrict__ new_k,
                       int len, int B, int N, float eps, int rows_per_split, int nmax,
-                      float* __restrict__ partial, float* __restrict__ norms) {
+                      float* __restrict__ partial, float* __restrict__ norms, int raw_anchor) {
     __shared__ float red[kStagedThreads / kLanesPerRow][kHeadDim + 4];
     const int u = blockIdx.y, s = blockIdx.x, splits = gridDim.x;
     const int n = len + B;
@@ -44,7 +44,7 @@ anchor_partial_kernel(const uint4* __restrict__ k_cache, const uint4* __restrict
         float x[16];
         unpack_row(a, b, x);
         const float r = sqrtf(row_sumsq(x));
-        const float inv = 1.0f / fmaxf(r, eps);
+        const float inv = raw_anchor ? 1.0f : 1.0f / fmaxf(r, eps);   // raw-mean anchor: the keys themselves are summed
         if (valid) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) acc[j] = fmaf(x[j], inv, acc[j]);
@@ -116,11 +116,14 @@ score_kernel(const uint4* __restrict__ k_cache, const uint4* __restrict__ new_k,
 __global__ void __launch_bounds__(kSelectThreads)
 select_kernel(const float* __restrict__ scores, int n, int N, int nmax, int len,
               int32_t* __restrict__ kept_idx, int32_t* __restrict__ first_evicted,
-              unsigned long long* __restrict__ moved_rows) {
+              unsigned long long* __restrict__ moved_rows, int window) {
     extern __shared__ uint32_t keys[];
     __shared__ SelectSmem sm;
     const int u = blockIdx.x, tid = threadIdx.x;
-    for (int i = tid; i < n; i += kSelectThreads) keys[i] = order_key(scores[static_cast<size_t>(u) * nmax + i]);
+    // sliding window (Sec. 3.2): the last `window` tokens carry the largest possible key, so the top-N
+    // selection keeps them all and fills the other N - window places by score
+    for (int i = tid; i < n; i += kSelectThreads)
+        keys[i] = i >= n - window ? 0xffffffffu : order_key(scores[static_cast<size_t>(u) * nmax + i]);
     if (tid == 0) sm.first_evicted = n;
     __syncthreads();
     const Threshold th = block_radix_select<kSelectThreads>(keys, n, N, sm);
