@@ -112,3 +112,31 @@ def test_bad_variant_arguments_are_rejected():
     with pytest.raises(KeyDiffError) as e:
         KeyDiff(1, 1, 2, 128, 64, 8, recent_window=-1)
     assert e.value.code == binding.KEYDIFF_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("mode,w", [(0, 0), (RAW, 900)])
+def test_fused_unit_beyond_the_register_select(mode, w):
+    # n = 9300 keys per unit: more than the 17 keys per thread the low-end select holds in registers,
+    # so the fused kernel takes its full-table select; two steps (the second on the running anchor)
+    U, N, B = 3, 9000, 300
+    k_cache, v_cache, stream = state(U, N, B, N, seed=77 + w, model="outlier")
+    kd = KeyDiff(1, 1, U, 128, N, B, path=binding.KEYDIFF_PATH_FUSED, anchor_mode=mode, recent_window=w)
+    kd.set_len(N)
+    for _ in range(2):
+        checked_step(kd, k_cache, v_cache, *stream.next_block(B), mode, w)
+    kd.close()
+
+
+def test_fused_crowded_threshold_bin_falls_back():
+    # thousands of identical keys: the threshold bin of the low-end select overflows and the kernel
+    # must take the exact-rank / radix route; ties keep the older tokens
+    U, N, B = 2, 2048, 128
+    k_cache, v_cache, stream = state(U, N, B, N, seed=5)
+    k_cache[:, 300:1900] = k_cache[:, 300:301]          # 1600 copies of one row
+    new_k, new_v = stream.next_block(B)
+    new_k[:, 10:90] = k_cache[:, 300:301]               # and 80 more in the block
+    kd = KeyDiff(1, 1, U, 128, N, B, path=binding.KEYDIFF_PATH_FUSED)
+    kd.set_len(N)
+    for _ in range(2):
+        checked_step(kd, k_cache, v_cache, new_k, new_v, 0, 0)
+    kd.close()
