@@ -219,9 +219,9 @@ def run_ours(args):
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": total_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16 in, fp32 arithmetic", "data": "synthetic",
+            "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "n_layers": wl.n_layers, "batch": wl.batch, "n_kv_heads": wl.n_kv_heads,
-                       "head_dim": d, "budget_N": N, "block_B": B, "units": U, "key_model": wl.key_model,
+                       "head_dim": d, "budget_N": N, "block_B": B, "units": U, "key_model": wl.key_model, "storage_dtype": "bf16",
                        "cache_bytes": 2 * U * N * d * 2, "l2_policy": "inputs larger than L2 (cache >> 126 MB)",
                        "path": "fused" if info["path"] == binding.KEYDIFF_PATH_FUSED else "staged",
                        "cluster_size": info["cluster_size"], "replicas": world},
