@@ -42,6 +42,14 @@
 //     the largest eviction score are kept among the first n - w, and the anchor is still formed
 //     from all n keys.
 //
+//   * unordered slot reuse (the *_slots entry point) -- Eq. (keydiff) gathers the kept rows but fixes
+//     no order for them (attention does not depend on the order of the cached pairs).  Reading: kept
+//     cache rows stay in their slots; the kept block rows, in block order, fill the freed slots (those
+//     of evicted cache rows and, while the cache is not full, the empty ones) in ascending slot
+//     order; a side array holds each slot's token position.  Candidates are numbered cache slots
+//     first, block rows after; equal scores keep the lower candidate number.  The sliding window is
+//     then defined on positions: tokens among the last w of the sequence are always kept.
+//
 // Every function is pinned by tests that do not call back into this file:
 // hand-worked examples, closed forms, the pairwise identity evaluated in numpy,
 // brute force over all subsets, and structural invariants.  No function here is
@@ -182,6 +190,67 @@ void evict_head(const HeadArgs& a) {
     if (a.m_out) *a.m_out = m;
 }
 
+// One unit with unordered slot reuse.  pos_in[len]: token position held by each valid slot;
+// the block rows are tokens next_pos .. next_pos + B - 1.  Outputs: the whole new cache
+// (k_out/v_out, N rows, the first min(N, len + B) slots valid), pos_out[N], src_out[N] = candidate
+// number (slot for a cache row, len + j for block row j) of what each valid slot now holds.
+struct SlotArgs {
+    const int64_t* pos_in; int64_t next_pos; int64_t* pos_out; int64_t* src_out;
+};
+void evict_head_slots(const HeadArgs& a, const SlotArgs& sa) {
+    const int64_t n = a.len + a.B, d = a.d, N = a.N;
+    auto k_row = [&](int64_t i) { return i < a.len ? a.k_cache + i * d : a.new_k + (i - a.len) * d; };
+    auto v_row = [&](int64_t i) { return i < a.len ? a.v_cache + i * d : a.new_v + (i - a.len) * d; };
+    auto pos_of = [&](int64_t i) { return i < a.len ? sa.pos_in[i] : sa.next_pos + (i - a.len); };
+    // the cache as it stands
+    for (int64_t i = 0; i < a.len; ++i) {
+        std::memcpy(a.k_out + i * d, k_row(i), d * sizeof(uint16_t));
+        std::memcpy(a.v_out + i * d, v_row(i), d * sizeof(uint16_t));
+        sa.pos_out[i] = sa.pos_in[i];
+        sa.src_out[i] = i;
+    }
+    std::vector<char> keep(n, 1);
+    double tau = 0.0, m = 0.0;
+    if (n > N) {
+        std::vector<double> K(static_cast<size_t>(n) * d), s(n), e(n);
+        for (int64_t i = 0; i < n; ++i)
+            for (int64_t c = 0; c < d; ++c) K[i * d + c] = bf16_bits_to_double(k_row(i)[c]);
+        scores_f64(K.data(), n, d, a.eps, nullptr, nullptr, &m, s.data(), a.anchor_mode);
+        for (int64_t i = 0; i < n; ++i) e[i] = eviction_score(s[i]);
+        if (a.e_out) std::copy(e.begin(), e.end(), a.e_out);
+        // the window: tokens among the last `window` positions of the sequence are kept whatever they score
+        const int64_t first_recent = sa.next_pos + a.B - a.window;
+        std::vector<int64_t> rest;            // candidates the score rule decides on, in candidate order
+        for (int64_t i = 0; i < n; ++i) if (pos_of(i) < first_recent) rest.push_back(i);
+        const int64_t in_window = n - static_cast<int64_t>(rest.size());
+        const int64_t quota = N - in_window;  // places left for them
+        std::vector<double> er(rest.size());
+        for (size_t j = 0; j < rest.size(); ++j) er[j] = e[rest[j]];
+        std::vector<int64_t> S(std::max<int64_t>(quota, 0));
+        const int64_t kept_rest = (quota > 0 && !rest.empty()) ? select_topn(er.data(), er.size(), quota, S.data(), &tau) : 0;
+        for (int64_t i : rest) keep[i] = 0;
+        for (int64_t j = 0; j < kept_rest; ++j) keep[rest[S[j]]] = 1;
+    }
+    // freed slots in ascending order take the kept block rows in block order
+    int64_t slot = 0;
+    auto next_free = [&]() {
+        while (slot < a.len && keep[slot]) ++slot;   // slots >= len are empty
+        return slot++;
+    };
+    for (int64_t j = 0; j < a.B; ++j) {
+        const int64_t i = a.len + j;
+        if (!keep[i]) continue;
+        const int64_t t = next_free();
+        std::memcpy(a.k_out + t * d, k_row(i), d * sizeof(uint16_t));
+        std::memcpy(a.v_out + t * d, v_row(i), d * sizeof(uint16_t));
+        sa.pos_out[t] = pos_of(i);
+        sa.src_out[t] = i;
+    }
+    if (a.len_out) *a.len_out = std::min(N, n);
+    if (a.tau_out) *a.tau_out = tau;
+    if (a.m_out) *a.m_out = m;
+}
+
 }  // namespace
 
 extern "C" {
@@ -294,6 +363,26 @@ void kd_oracle_evict_units_bf16_ex(const uint16_t* k_cache, const uint16_t* v_ca
         a.anchor_mode = anchor_mode;
         a.window = window;
         evict_head(a);
+    }
+}
+
+// U units with unordered slot reuse (single-threaded per call).  pos_in/pos_out/src_out: [U][N];
+// e_out [U][len+B] (written only when an eviction happens); the other layouts as above.
+void kd_oracle_evict_units_bf16_slots(const uint16_t* k_cache, const uint16_t* v_cache, const int64_t* pos_in,
+                                      int64_t len, int64_t next_pos,
+                                      const uint16_t* new_k, const uint16_t* new_v, int64_t B,
+                                      int64_t N, int64_t d, double eps, int64_t U, int32_t anchor_mode, int64_t window,
+                                      uint16_t* k_out, uint16_t* v_out, int64_t* pos_out, int64_t* src_out,
+                                      double* e_out, double* tau_out, double* m_out) {
+    const int64_t n = len + B;
+    for (int64_t u = 0; u < U; ++u) {
+        HeadArgs a{k_cache + u * N * d, v_cache + u * N * d, len, new_k + u * B * d, new_v + u * B * d, B, N, d, eps,
+                   k_out + u * N * d, v_out + u * N * d, nullptr,
+                   e_out ? e_out + u * n : nullptr, nullptr,
+                   tau_out ? tau_out + u : nullptr, m_out ? m_out + u : nullptr};
+        a.anchor_mode = anchor_mode;
+        a.window = window;
+        evict_head_slots(a, SlotArgs{pos_in + u * N, next_pos, pos_out + u * N, src_out + u * N});
     }
 }
 

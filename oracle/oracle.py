@@ -63,6 +63,9 @@ def _load():
         lib.kd_oracle_evict_units_bf16_ex.argtypes = [c_hp, c_hp, i64, c_hp, c_hp, i64, i64, i64, f64, i64,
                                                       ctypes.c_int32, i64, c_hp, c_hp, c_dp, c_ip, c_dp, c_dp]
         lib.kd_oracle_evict_units_bf16_ex.restype = None
+        lib.kd_oracle_evict_units_bf16_slots.argtypes = [c_hp, c_hp, c_ip, i64, i64, c_hp, c_hp, i64, i64, i64, f64, i64,
+                                                         ctypes.c_int32, i64, c_hp, c_hp, c_ip, c_ip, c_dp, c_dp, c_dp]
+        lib.kd_oracle_evict_units_bf16_slots.restype = None
         _lib = lib
     return _lib
 
@@ -162,3 +165,46 @@ def evict_units_bf16(k_cache, v_cache, length: int, new_k, new_v, N: int,
             list(pool.map(run, range(used)))
     return {"k": k_out, "v": v_out, "len": keep, "e": e if n > N else None,
             "S": S_full[:, :keep].copy(), "tau": tau, "m": m, "threads": int(used)}
+
+
+def evict_units_bf16_slots(k_cache, v_cache, pos, length: int, next_pos: int, new_k, new_v, N: int,
+                           eps: float = DEFAULT_EPS, n_threads: int = 1, anchor_mode: int = 0, recent_window: int = 0):
+    """U units with unordered slot reuse: kept cache rows stay in their slots, kept block rows fill
+    the freed slots.  pos: (U, N) int64, the token position held by each of the `length` valid slots;
+    the block rows are tokens next_pos .. next_pos + B - 1.
+
+    Returns dict: k, v (U, N, d) uint16, pos (U, N) int64, src (U, N) int64 (candidate number now in
+    each slot: the slot itself for a cache row, length + j for block row j), len, e (U, n) or None,
+    tau, m, threads.
+    """
+    k_cache = np.ascontiguousarray(k_cache, dtype=np.uint16)
+    v_cache = np.ascontiguousarray(v_cache, dtype=np.uint16)
+    new_k = np.ascontiguousarray(new_k, dtype=np.uint16)
+    new_v = np.ascontiguousarray(new_v, dtype=np.uint16)
+    pos = np.ascontiguousarray(pos, dtype=np.int64)
+    U, cap, d = k_cache.shape
+    B = new_k.shape[1]
+    assert cap == N and v_cache.shape == k_cache.shape and pos.shape == (U, N)
+    assert new_k.shape == (U, B, d) and new_v.shape == (U, B, d)
+    assert 0 <= length <= N and 0 <= recent_window <= N
+    n = length + B
+    k_out = np.zeros((U, N, d), dtype=np.uint16)
+    v_out = np.zeros((U, N, d), dtype=np.uint16)
+    pos_out = np.zeros((U, N), dtype=np.int64)
+    src = np.zeros((U, N), dtype=np.int64)
+    e = np.zeros((U, n), dtype=np.float64)
+    tau, m = np.zeros(U), np.zeros(U)
+    from concurrent.futures import ThreadPoolExecutor
+    used = max(1, min(n_threads, U))
+    lib = _load()
+
+    def run(t):
+        for u in range(t, U, used):
+            lib.kd_oracle_evict_units_bf16_slots(
+                _hp(k_cache[u]), _hp(v_cache[u]), _ip(pos[u]), length, next_pos, _hp(new_k[u]), _hp(new_v[u]),
+                B, N, d, eps, 1, anchor_mode, recent_window, _hp(k_out[u]), _hp(v_out[u]), _ip(pos_out[u]),
+                _ip(src[u]), _dp(e[u]), _dp(tau[u:u + 1]), _dp(m[u:u + 1]))
+    with ThreadPoolExecutor(used) as pool:
+        list(pool.map(run, range(used)))
+    return {"k": k_out, "v": v_out, "pos": pos_out, "src": src, "len": min(N, n), "e": e if n > N else None,
+            "tau": tau, "m": m, "threads": int(used)}
