@@ -69,6 +69,15 @@ enum {
     KEYDIFF_ANCHOR_RAW_MEAN = 1     /* mu = (1/n) sum_i k_i */
 };
 
+/* Where the kept rows end up.  Eq. (keydiff) gathers them, K' = gather(K,S), without fixing their
+ * order (attention does not depend on the order of the cached pairs; positions are already rotated
+ * into the keys).  Both layouts are built. */
+enum {
+    KEYDIFF_COMPACT_ORDERED = 0,    /* kept rows in original token order, compacted to the front (default) */
+    KEYDIFF_COMPACT_SLOT_REUSE = 1  /* kept cache rows stay in their slots; the kept block rows take the
+                                       freed slots: at most block_B rows per tensor are written */
+};
+
 /* Which kernels serve keydiff_evict. */
 enum {
     KEYDIFF_PATH_AUTO = 0,    /* fused cluster kernel when a unit fits, else the staged kernels */
@@ -91,6 +100,7 @@ typedef struct {
     int32_t anchor_mode;   /* KEYDIFF_ANCHOR_*: which mean is the anchor (Sec. 3.2) */
     int32_t recent_window; /* w >= 0 most recent tokens that are never evicted (Sec. 3.2, "KeyDiff with
                               sliding window"); 0 = plain KeyDiff; w <= budget */
+    int32_t compaction;    /* KEYDIFF_COMPACT_*: layout of the kept rows */
 } keydiff_config;
 
 /*
@@ -99,7 +109,7 @@ typedef struct {
  * partials, per-unit counters, one status word).  Synchronous.  *out is set only on
  * KEYDIFF_OK.  The initial cache length is 0 (C_0 = empty, Eq. block_processing).
  * Errors: INVALID_ARG (NULL, non-positive sizes, unknown anchor_mode, recent_window outside
- * [0, budget]), UNSUPPORTED (dtype, head_dim, a unit
+ * [0, budget], unknown compaction), UNSUPPORTED (dtype, head_dim, a unit
  * too large for the requested path, no sm_100 device), ALLOC, CUDA.
  */
 KEYDIFF_API int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out);
@@ -117,6 +127,13 @@ KEYDIFF_API int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out);
  *   With recent_window = w > 0 (Sec. 3.2, sliding window; the paper gives no formula, this is the
  *   reading taken): the last w of the n tokens are always kept, the N - w tokens with the largest e are
  *   kept among the first n - w, and the anchor is still formed from all n keys.
+ *   With compaction = KEYDIFF_COMPACT_SLOT_REUSE the n candidates are numbered slots 0 .. len-1 first,
+ *   block rows len .. n-1 after; scores and selection are the same (ties: lower candidate number wins);
+ *   kept cache rows are not touched, and the kept block rows, in block order, are written into the freed
+ *   slots (those of evicted cache rows, then slots >= len that were still empty) in ascending slot
+ *   order.  The ctx keeps each slot's token position (keydiff_get_positions); the sliding window then
+ *   means the tokens at the last w positions of the sequence.  An append-only step is the same as in
+ *   the ordered layout.
  * k_cache, v_cache: device, in/out, caller-owned.  new_k, new_v: device, read only,
  * caller-owned; they may be reused once the work enqueued on `stream` has completed.
  * budget_N, n_kv_heads, head_dim restate the ctx's values and must equal them;
@@ -185,6 +202,17 @@ KEYDIFF_API int keydiff_set_len(keydiff_ctx* ctx, int32_t len);
  */
 KEYDIFF_API int keydiff_get_scratch(const keydiff_ctx* ctx, const float** scores, const int32_t** kept_idx,
                         const int32_t** first_evicted, const int32_t** status);
+
+/*
+ * keydiff_get_positions -- slot reuse only (else KEYDIFF_ERR_STATE): device pointer to pos[U][N] int32,
+ * the token position (0-based index in the sequence) held by each of the first len slots, valid once
+ * the stream work of the latest step has completed, and the position the next new token will get.
+ * keydiff_set_len(len) declares slots 0 .. len-1 to hold tokens 0 .. len-1; keydiff_reset starts a new
+ * sequence.  In this mode kept_idx[u][s] (keydiff_get_scratch) is the candidate number slot s now holds
+ * (s itself for a cache row that stayed, len + j for block row j), and the moved-rows counter counts
+ * the block rows written.  Either output pointer may be NULL.
+ */
+KEYDIFF_API int keydiff_get_positions(const keydiff_ctx* ctx, const int32_t** pos, long long* next_pos);
 
 /*
  * keydiff_get_moved_rows -- device pointer to a 64-bit counter: the number of kept rows (per

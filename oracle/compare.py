@@ -90,3 +90,79 @@ def check_step(k_cache, v_cache, length, new_k, new_v, N, gpu_k, gpu_v, gpu_scor
         if (S_gpu == S_ref).all():
             assert (gpu_k[u, :N] == ref["k"][j]).all() and (gpu_v[u, :N] == ref["v"][j]).all()
     return rep
+
+
+def check_step_slots(k_cache, v_cache, pos, next_pos, length, new_k, new_v, N, gpu_k, gpu_v, gpu_scores, gpu_src,
+                     gpu_pos, eps=oracle.DEFAULT_EPS, units=None, n_threads=1, anchor_mode=0, recent_window=0):
+    """The same acceptance rules for a step with unordered slot reuse.  pos: int [U, N] token positions of
+    the slots before the step; gpu_src: int32 [U, N], the candidate number each slot holds after it (the
+    library's kept_idx in this mode); gpu_pos: int32 [U, N] positions after it.
+      scores     as in check_step;
+      selection  the kept candidates are the top-N of the GPU's own fp32 scores under (e desc, candidate
+                 number asc), tokens at the last recent_window positions always kept; agreement with the
+                 oracle outside the tau band;
+      placement  kept cache rows untouched; the kept block rows, in block order, in the freed slots in
+                 ascending order; rows bit-exact; positions exact."""
+    U = k_cache.shape[0]
+    sel = np.arange(U) if units is None else np.asarray(units)
+    B = new_k.shape[1]
+    n = length + B
+    assert n > N, "check_step_slots is for evicting steps"
+    ref = oracle.evict_units_bf16_slots(k_cache[sel], v_cache[sel], pos[sel], length, next_pos, new_k[sel], new_v[sel], N,
+                                        eps, n_threads, anchor_mode=anchor_mode, recent_window=recent_window)
+    rep = {"units": len(sel), "n": n, "max_score_err_over_tol": 0.0, "max_plain_rel": 0.0,
+           "set_mismatch_in_band": 0, "min_anchor_norm": float(ref["m"].min())}
+    for j, u in enumerate(sel):
+        allk = np.concatenate([k_cache[u, :length], new_k[u]])
+        allv = np.concatenate([v_cache[u, :length], new_v[u]])
+        cand_pos = np.concatenate([pos[u, :length].astype(np.int64), next_pos + np.arange(B)])
+        e_ref = ref["e"][j]
+        e_gpu = gpu_scores[u, :n].astype(np.float64)
+        assert np.isfinite(e_gpu).all(), f"unit {u}: non-finite GPU score"
+        if ref["m"][j] >= MIN_ANCHOR_NORM:
+            K = _bf16_to_f64(allk)
+            r = np.sqrt((K * K).sum(1))
+            unit = K if anchor_mode == 1 else K / np.maximum(r, eps)[:, None]
+            mu = unit.sum(0) / n
+            kappa = (np.abs(K) @ np.abs(mu)) / np.maximum(np.sqrt((mu * mu).sum()) * r, eps)
+            tol = SCORE_RTOL * np.maximum(np.abs(e_ref), kappa)
+            err = np.abs(e_gpu - e_ref)
+            worst = float((err / np.maximum(tol, 1e-300)).max())
+            rep["max_score_err_over_tol"] = max(rep["max_score_err_over_tol"], worst)
+            assert worst <= 1.0, f"unit {u}: score error {worst:.3f}x the tolerance"
+            big = np.abs(e_ref) >= PLAIN_REL_FLOOR
+            if big.any():
+                rel = float((err[big] / np.abs(e_ref[big])).max())
+                rep["max_plain_rel"] = max(rep["max_plain_rel"], rel)
+                assert rel <= SCORE_RTOL, f"unit {u}: plain relative score error {rel:.3e}"
+        # ---- selection w.r.t. the GPU's own scores
+        src = gpu_src[u].astype(np.int64)
+        assert len(set(src.tolist())) == N and src.min() >= 0 and src.max() < n, f"unit {u}: slots do not hold N distinct candidates"
+        recent = cand_pos >= next_pos + B - recent_window
+        rest = np.nonzero(~recent)[0]
+        e32 = gpu_scores[u, :n]
+        order = rest[np.lexsort((rest, -e32[rest].astype(np.float64)))]
+        want = np.sort(np.concatenate([order[:max(N - int(recent.sum()), 0)], np.nonzero(recent)[0]]))
+        S_gpu = np.sort(src)
+        assert (S_gpu == want).all(), f"unit {u}: kept candidates are not the top-N of the GPU's own scores"
+        # ---- agreement with the oracle outside the threshold band
+        S_ref = np.sort(ref["src"][j])
+        if not (S_gpu == S_ref).all():
+            diff = np.setxor1d(S_gpu, S_ref)
+            dist = np.abs(e_ref[diff] - ref["tau"][j])
+            assert (dist <= TAU_BAND).all(), f"unit {u}: kept sets differ on candidates {diff[dist > TAU_BAND][:8]} outside the tau band"
+            rep["set_mismatch_in_band"] += len(diff)
+        # ---- placement, given the kept set
+        kept = np.zeros(n, dtype=bool); kept[S_gpu] = True
+        free = np.concatenate([np.nonzero(~kept[:length])[0], np.arange(length, N)])
+        blocks = length + np.nonzero(kept[length:])[0]
+        assert len(free) == len(blocks)
+        exp_src = np.arange(N); exp_src[free] = blocks
+        assert (src == exp_src).all(), f"unit {u}: block rows are not in the freed slots in order"
+        assert (gpu_pos[u].astype(np.int64) == cand_pos[exp_src]).all(), f"unit {u}: slot positions are wrong"
+        assert (gpu_k[u, :N] == allk[exp_src]).all(), f"unit {u}: K rows are not bit-exact copies"
+        assert (gpu_v[u, :N] == allv[exp_src]).all(), f"unit {u}: V rows are not bit-exact copies"
+        if (S_gpu == S_ref).all():
+            assert (gpu_k[u, :N] == ref["k"][j]).all() and (gpu_v[u, :N] == ref["v"][j]).all()
+            assert (gpu_pos[u] == ref["pos"][j]).all()
+    return rep

@@ -21,11 +21,12 @@ KEYDIFF_ERR_TOO_LARGE = -7
 KEYDIFF_BF16 = 0
 KEYDIFF_PATH_AUTO, KEYDIFF_PATH_STAGED, KEYDIFF_PATH_FUSED = 0, 1, 2
 KEYDIFF_ANCHOR_NORMALISED, KEYDIFF_ANCHOR_RAW_MEAN = 0, 1
+KEYDIFF_COMPACT_ORDERED, KEYDIFF_COMPACT_SLOT_REUSE = 0, 1
 
 # every symbol include/keydiff.h declares
 EXPORTS = ["keydiff_create", "keydiff_evict", "keydiff_evict_host", "keydiff_destroy", "keydiff_reset",
            "keydiff_get_len", "keydiff_set_len", "keydiff_get_scratch", "keydiff_get_moved_rows",
-           "keydiff_get_launch_info", "keydiff_evict_static", "keydiff_set_incremental",
+           "keydiff_get_launch_info", "keydiff_evict_static", "keydiff_set_incremental", "keydiff_get_positions",
            "keydiff_strerror", "keydiff_last_cuda_error"]
 
 
@@ -33,7 +34,8 @@ class keydiff_config(ctypes.Structure):
     _fields_ = [("n_layers", ctypes.c_int32), ("batch", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("budget", ctypes.c_int32), ("max_block", ctypes.c_int32),
                 ("dtype", ctypes.c_int32), ("path", ctypes.c_int32), ("eps", ctypes.c_float),
-                ("device", ctypes.c_int32), ("anchor_mode", ctypes.c_int32), ("recent_window", ctypes.c_int32)]
+                ("device", ctypes.c_int32), ("anchor_mode", ctypes.c_int32), ("recent_window", ctypes.c_int32),
+                ("compaction", ctypes.c_int32)]
 
 
 class KeyDiffError(RuntimeError):
@@ -66,6 +68,7 @@ def load_library() -> ctypes.CDLL:
     lib.keydiff_set_incremental.argtypes = [vp, i32]
     lib.keydiff_get_scratch.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.keydiff_get_moved_rows.argtypes = [vp, ctypes.POINTER(vp)]
+    lib.keydiff_get_positions.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_longlong)]
     lib.keydiff_get_launch_info.argtypes = [vp, i32p, i32p, i32p]
     lib.keydiff_evict_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, ctypes.c_float, vp]
     lib.keydiff_strerror.argtypes = [ctypes.c_int]
@@ -101,13 +104,14 @@ class KeyDiff:
 
     def __init__(self, n_layers: int, batch: int, n_kv_heads: int, head_dim: int, budget: int, max_block: int,
                  *, path: int = KEYDIFF_PATH_AUTO, eps: float = 0.0, device: int | None = None,
-                 anchor_mode: int = KEYDIFF_ANCHOR_NORMALISED, recent_window: int = 0):
+                 anchor_mode: int = KEYDIFF_ANCHOR_NORMALISED, recent_window: int = 0,
+                 compaction: int = KEYDIFF_COMPACT_ORDERED):
         self._lib = load_library()
         self._ctx = ctypes.c_void_p()
         if device is None:
             device = torch.cuda.current_device() if torch.cuda.is_available() else 0
         self.cfg = keydiff_config(n_layers, batch, n_kv_heads, head_dim, budget, max_block, KEYDIFF_BF16, path,
-                                  eps, device, anchor_mode, recent_window)
+                                  eps, device, anchor_mode, recent_window, compaction)
         _check(self._lib.keydiff_create(ctypes.byref(self.cfg), ctypes.byref(self._ctx)))
         self.units = n_layers * batch * n_kv_heads
         self.budget, self.max_block, self.head_dim, self.n_kv_heads = budget, max_block, head_dim, n_kv_heads
@@ -175,6 +179,12 @@ class KeyDiff:
         mk = lambda ptr, shape, ts: torch.as_tensor(_DevArray(ptr.value, shape, ts), device=self.device)
         return {"scores": mk(p[0], (U, nmax), "<f4"), "kept_idx": mk(p[1], (U, N), "<i4"),
                 "first_evicted": mk(p[2], (U,), "<i4"), "status": mk(p[3], (1,), "<i4")}
+
+    def positions(self):
+        """``keydiff_get_positions`` (slot reuse only): (view of pos [U, N] int32, next position)."""
+        p, nxt = ctypes.c_void_p(), ctypes.c_longlong()
+        _check(self._lib.keydiff_get_positions(self._ctx, ctypes.byref(p), ctypes.byref(nxt)))
+        return torch.as_tensor(_DevArray(p.value, (self.units, self.budget), "<i4"), device=self.device), nxt.value
 
     def moved_rows(self) -> int:
         """Cumulative count of kept rows that changed position (synchronises the device)."""

@@ -59,6 +59,10 @@ struct keydiff_ctx {
     int32_t* first_evicted = nullptr; // [U]
     int32_t* status = nullptr;        // [1]
     unsigned long long* moved_rows = nullptr;   // [1] cumulative count of rows that changed position
+    // unordered slot reuse: token position held by every slot, and the position of the next new token
+    int32_t* pos = nullptr;           // [U][N]
+    long long next_pos = 0;
+    bool pos_stale = true;            // pos must be reset to the identity before the next step uses it
     void* stage_k = nullptr;          // [U][max_block][128] bf16, keydiff_evict_host only
     void* stage_v = nullptr;
 };
@@ -68,7 +72,7 @@ namespace {
 void free_scratch(keydiff_ctx* c) {
     cudaFree(c->partial); cudaFree(c->norms); cudaFree(c->scores); cudaFree(c->kept_idx);
     cudaFree(c->first_evicted); cudaFree(c->status); cudaFree(c->moved_rows); cudaFree(c->stage_k); cudaFree(c->stage_v);
-    cudaFree(c->anchor_sum[0]); cudaFree(c->anchor_sum[1]); cudaFree(c->anchor_delta);
+    cudaFree(c->anchor_sum[0]); cudaFree(c->anchor_sum[1]); cudaFree(c->anchor_delta); cudaFree(c->pos);
 }
 
 int check_step_args(const keydiff_ctx* ctx, const void* k_cache, const void* v_cache,
@@ -83,6 +87,8 @@ int check_step_args(const keydiff_ctx* ctx, const void* k_cache, const void* v_c
     if (dev != ctx->cfg.device) return KEYDIFF_ERR_STATE;   // the ctx's device must be current
     return KEYDIFF_OK;
 }
+
+inline bool slot_reuse(const keydiff_ctx* c) { return c->cfg.compaction == KEYDIFF_COMPACT_SLOT_REUSE; }
 
 using FusedKernel = void (*)(kd::FusedParams);
 
@@ -216,8 +222,13 @@ int launch_staged(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const u
     score_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, c->len, B, N, c->eps, rows_per_split, c->nmax,
                                                   c->partial, c->norms, c->scores);
     select_kernel<<<U, kSelectThreads, static_cast<size_t>(n) * 4, st>>>(c->scores, n, N, c->nmax, c->len, c->kept_idx,
-                                                                          c->first_evicted, c->moved_rows, c->cfg.recent_window);
-    compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, c->len, B, N, c->kept_idx, c->first_evicted);
+                                                                          c->first_evicted, c->moved_rows, c->cfg.recent_window,
+                                                                          slot_reuse(c) ? c->pos : nullptr, static_cast<int>(c->next_pos));
+    if (slot_reuse(c))
+        slot_place_kernel<<<U, kCompactThreads, static_cast<size_t>(B) * 8, st>>>(kc, vc, nk, nv, c->len, B, N, c->kept_idx, c->pos,
+                                                                                  static_cast<int>(c->next_pos), c->moved_rows);
+    else
+        compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, c->len, B, N, c->kept_idx, c->first_evicted);
     KD_CUDA(cudaGetLastError());
     return KEYDIFF_OK;
 }
@@ -235,11 +246,13 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
         return KEYDIFF_ERR_INVALID_ARG;
     if (cfg->anchor_mode != KEYDIFF_ANCHOR_NORMALISED && cfg->anchor_mode != KEYDIFF_ANCHOR_RAW_MEAN) return KEYDIFF_ERR_INVALID_ARG;
     if (cfg->recent_window < 0 || cfg->recent_window > cfg->budget) return KEYDIFF_ERR_INVALID_ARG;
+    if (cfg->compaction != KEYDIFF_COMPACT_ORDERED && cfg->compaction != KEYDIFF_COMPACT_SLOT_REUSE) return KEYDIFF_ERR_INVALID_ARG;
     if (cfg->dtype != KEYDIFF_BF16 || cfg->head_dim != kd::kHeadDim) return KEYDIFF_ERR_UNSUPPORTED;
     const long long U = 1LL * cfg->n_layers * cfg->batch * cfg->n_kv_heads;
     const long long nmax = 1LL * cfg->budget + cfg->max_block;
     if (U > 65535 || nmax > (1 << 30)) return KEYDIFF_ERR_UNSUPPORTED;   // gridDim.y limit of the staged kernels
     if (nmax * 4 > kMaxSelectSmem) return KEYDIFF_ERR_UNSUPPORTED;
+    if (cfg->compaction == KEYDIFF_COMPACT_SLOT_REUSE && 8LL * cfg->max_block > kMaxSelectSmem) return KEYDIFF_ERR_UNSUPPORTED;
 
     int count = 0;
     KD_CUDA(cudaGetDeviceCount(&count));
@@ -282,9 +295,15 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
         ok = cudaFuncSetAttribute(kd::select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   kMaxSelectSmem) == cudaSuccess;
     }
+    if (ok && cfg->compaction == KEYDIFF_COMPACT_SLOT_REUSE) {
+        ok = cudaMalloc(&c->pos, sizeof(int32_t) * U * cfg->budget) == cudaSuccess &&
+             cudaMemset(c->pos, 0, sizeof(int32_t) * U * cfg->budget) == cudaSuccess &&
+             cudaFuncSetAttribute(kd::slot_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  std::max(48 * 1024, 8 * cfg->max_block)) == cudaSuccess;
+    }
     if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
     if (ok && cfg->path != KEYDIFF_PATH_STAGED) {
-        if (plan_fused(c, prop.multiProcessorCount)) {
+        if (!slot_reuse(c) && plan_fused(c, prop.multiProcessorCount)) {
             c->path = KEYDIFF_PATH_FUSED;
             const size_t sum_bytes = sizeof(double) * U * kd::kHeadDim;
             ok = cudaMalloc(&c->anchor_sum[0], sum_bytes) == cudaSuccess && cudaMalloc(&c->anchor_sum[1], sum_bytes) == cudaSuccess &&
@@ -322,13 +341,26 @@ int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache, const void* ne
     const uint4* nk = static_cast<const uint4*>(new_k);
     const uint4* nv = static_cast<const uint4*>(new_v);
     const int N = ctx->cfg.budget, n = ctx->len + block_B;
+    if (slot_reuse(ctx)) {
+        if (ctx->next_pos + block_B > 0x7fffffffLL) return KEYDIFF_ERR_STATE;   // positions are int32
+        if (ctx->pos_stale) {
+            // the cache as the caller declared it: slot s holds token s
+            const int total = ctx->U * N;
+            kd::pos_iota_kernel<<<(total + 255) / 256, 256, 0, st>>>(ctx->pos, N, total);
+            ctx->pos_stale = false;
+        }
+    }
     if (n <= N) {
         // Sec. 2.3: the budget is not exceeded, nothing is evicted
         const int threads = 256;
         const dim3 grid((block_B * kd::kRowVec + threads - 1) / threads, ctx->U, 2);
         kd::append_kernel<<<grid, threads, 0, st>>>(kc, vc, nk, nv, ctx->len, block_B, N);
+        if (slot_reuse(ctx))
+            kd::pos_append_kernel<<<dim3((block_B + threads - 1) / threads, ctx->U), threads, 0, st>>>(
+                ctx->pos, ctx->len, block_B, N, static_cast<int>(ctx->next_pos));
         KD_CUDA(cudaGetLastError());
         ctx->len = n;
+        ctx->next_pos += block_B;
         ctx->anchor_valid = false;   // the appended rows are not in the running anchor
         return KEYDIFF_OK;
     }
@@ -336,6 +368,7 @@ int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache, const void* ne
                                                     : launch_staged(ctx, kc, vc, nk, nv, block_B, st);
     if (lrc != KEYDIFF_OK) return lrc;
     ctx->len = N;
+    ctx->next_pos += block_B;
     return KEYDIFF_OK;
 }
 
@@ -384,6 +417,8 @@ int keydiff_reset(keydiff_ctx* ctx) {
     if (!ctx) return KEYDIFF_ERR_INVALID_ARG;
     ctx->len = 0;
     ctx->anchor_valid = false;
+    ctx->next_pos = 0;
+    ctx->pos_stale = true;
     return KEYDIFF_OK;
 }
 
@@ -403,6 +438,8 @@ int keydiff_set_len(keydiff_ctx* ctx, int32_t len) {
     if (!ctx || len < 0 || len > ctx->cfg.budget) return KEYDIFF_ERR_INVALID_ARG;
     ctx->len = len;
     ctx->anchor_valid = false;   // the caller brought its own cache contents
+    ctx->next_pos = len;         // ... which are tokens 0 .. len-1 in token order
+    ctx->pos_stale = true;
     return KEYDIFF_OK;
 }
 
@@ -413,6 +450,14 @@ int keydiff_get_scratch(const keydiff_ctx* ctx, const float** scores, const int3
     if (kept_idx) *kept_idx = ctx->kept_idx;
     if (first_evicted) *first_evicted = ctx->first_evicted;
     if (status) *status = ctx->status;
+    return KEYDIFF_OK;
+}
+
+int keydiff_get_positions(const keydiff_ctx* ctx, const int32_t** pos, long long* next_pos) {
+    if (!ctx) return KEYDIFF_ERR_INVALID_ARG;
+    if (!slot_reuse(ctx)) return KEYDIFF_ERR_STATE;
+    if (pos) *pos = ctx->pos;
+    if (next_pos) *next_pos = ctx->next_pos;
     return KEYDIFF_OK;
 }
 
@@ -548,7 +593,7 @@ extern "C" int keydiff_evict_static(void* k_cache, void* v_cache, const void* ne
     const dim3 grid(splits, U);
     anchor_partial_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, len, block_B, N, e, rows_per_split, nn, partial, norms, 0);
     score_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, len, block_B, N, e, rows_per_split, nn, partial, norms, scores);
-    select_kernel<<<U, kSelectThreads, static_cast<size_t>(nn) * 4, st>>>(scores, nn, N, nn, len, kept, first, moved, 0);
+    select_kernel<<<U, kSelectThreads, static_cast<size_t>(nn) * 4, st>>>(scores, nn, N, nn, len, kept, first, moved, 0, nullptr, 0);
     compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, len, block_B, N, kept, first);
     KD_CUDA(cudaGetLastError());
     return KEYDIFF_OK;

@@ -116,14 +116,20 @@ score_kernel(const uint4* __restrict__ k_cache, const uint4* __restrict__ new_k,
 __global__ void __launch_bounds__(kSelectThreads)
 select_kernel(const float* __restrict__ scores, int n, int N, int nmax, int len,
               int32_t* __restrict__ kept_idx, int32_t* __restrict__ first_evicted,
-              unsigned long long* __restrict__ moved_rows, int window) {
+              unsigned long long* __restrict__ moved_rows, int window,
+              const int32_t* __restrict__ pos, int next_pos) {
     extern __shared__ uint32_t keys[];
     __shared__ SelectSmem sm;
     const int u = blockIdx.x, tid = threadIdx.x;
     // sliding window (Sec. 3.2): the last `window` tokens carry the largest possible key, so the top-N
-    // selection keeps them all and fills the other N - window places by score
-    for (int i = tid; i < n; i += kSelectThreads)
-        keys[i] = i >= n - window ? 0xffffffffu : order_key(scores[static_cast<size_t>(u) * nmax + i]);
+    // selection keeps them all and fills the other N - window places by score.  With slot reuse (pos !=
+    // nullptr) the cache is not in token order and "last" is read off the slots' token positions.
+    const int first_recent = next_pos + (n - len) - window;
+    for (int i = tid; i < n; i += kSelectThreads) {
+        const bool recent = pos ? (i < len ? pos[static_cast<size_t>(u) * N + i] : next_pos + (i - len)) >= first_recent
+                                : i >= n - window;
+        keys[i] = recent ? 0xffffffffu : order_key(scores[static_cast<size_t>(u) * nmax + i]);
+    }
     if (tid == 0) sm.first_evicted = n;
     __syncthreads();
     const Threshold th = block_radix_select<kSelectThreads>(keys, n, N, sm);
@@ -149,7 +155,8 @@ select_kernel(const float* __restrict__ scores, int n, int N, int nmax, int len,
     if (tid == 0) {
         first_evicted[u] = sm.first_evicted;
         // block rows always move into the cache, cache rows only from the first evicted one on
-        atomicAdd(moved_rows, static_cast<unsigned long long>(N - min(len, sm.first_evicted)));
+        // (with slot reuse the placement kernel counts the rows it writes)
+        if (!pos) atomicAdd(moved_rows, static_cast<unsigned long long>(N - min(len, sm.first_evicted)));
     }
 }
 
@@ -180,6 +187,65 @@ compact_kernel(uint4* k_cache, uint4* v_cache,     // read and written here: no 
         for (int q = threadIdx.x; q < cnt; q += kCompactThreads) dst[q] = stage[q];
         __syncthreads();
     }
+}
+
+// Step a4 with unordered slot reuse (Eq. (keydiff) gathers the kept rows without fixing their order):
+// kept cache rows stay where they are; the kept block rows, in block order, take the freed slots
+// (evicted cache rows, then slots >= len that were still empty) in ascending slot order.  Input:
+// kept[u][0..N) = ascending candidate numbers of the kept tokens (slots first, block rows after).
+// Output: the rows, pos[u][slot] = token position, and kept[u][slot] rewritten to the candidate
+// number each slot now holds.  grid = U, dynamic smem = 8 * B bytes.
+__global__ void __launch_bounds__(kCompactThreads)
+slot_place_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
+                  const uint4* __restrict__ new_k, const uint4* __restrict__ new_v,
+                  int len, int B, int N, int32_t* __restrict__ kept, int32_t* __restrict__ pos, int next_pos,
+                  unsigned long long* __restrict__ moved_rows) {
+    extern __shared__ int32_t place[];   // slot_of[B], block_of[B]: the r-th freed slot, the r-th kept block row
+    __shared__ int kc_sh;
+    int32_t* slot_of = place;
+    int32_t* block_of = place + B;
+    const int u = blockIdx.x, tid = threadIdx.x;
+    int32_t* L = kept + static_cast<size_t>(u) * N;
+    // kc = kept cache rows = entries below len (L ascends): the one position where the list crosses len
+    if (tid == 0) kc_sh = N;
+    __syncthreads();
+    for (int j = tid; j < N; j += kCompactThreads)
+        if (L[j] >= len && (j == 0 || L[j - 1] < len)) kc_sh = j;
+    __syncthreads();
+    const int kc = kc_sh, kb = N - kc;   // kb kept block rows = kb freed slots
+    for (int r = tid; r < kb; r += kCompactThreads) block_of[r] = L[kc + r] - len;
+    // a slot s missing between L[j-1] and L[j] has j kept slots below it: it is freed slot number s - j
+    for (int j = tid; j <= kc; j += kCompactThreads) {
+        const int lo = j == 0 ? 0 : L[j - 1] + 1, hi = j == kc ? len : L[j];
+        for (int sl = lo; sl < hi; ++sl) slot_of[sl - j] = sl;
+    }
+    for (int sl = len + tid; sl < N; sl += kCompactThreads) slot_of[sl - kc] = sl;   // the empty slots
+    __syncthreads();
+    for (int sl = tid; sl < N; sl += kCompactThreads) L[sl] = sl;
+    __syncthreads();
+    for (int r = tid; r < kb; r += kCompactThreads) {
+        L[slot_of[r]] = len + block_of[r];
+        pos[static_cast<size_t>(u) * N + slot_of[r]] = next_pos + block_of[r];
+    }
+    for (int q = tid; q < kb * kRowVec; q += kCompactThreads) {
+        const int r = q >> 4, c = q & 15;
+        const size_t dst = (static_cast<size_t>(u) * N + slot_of[r]) * kRowVec + c;
+        const size_t src = (static_cast<size_t>(u) * B + block_of[r]) * kRowVec + c;
+        k_cache[dst] = new_k[src];
+        v_cache[dst] = new_v[src];
+    }
+    if (tid == 0) atomicAdd(moved_rows, static_cast<unsigned long long>(kb));
+}
+
+// Token positions of the slots: identity (a cache the caller filled in token order) ...
+__global__ void pos_iota_kernel(int32_t* __restrict__ pos, int N, int total) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < total) pos[i] = i % N;
+}
+// ... and those of appended block rows: slot len + j holds token next_pos + j.  grid = (ceil(B/threads), U).
+__global__ void pos_append_kernel(int32_t* __restrict__ pos, int len, int B, int N, int next_pos) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < B) pos[static_cast<size_t>(blockIdx.y) * N + len + j] = next_pos + j;
 }
 
 // Step a0 when the budget is not exceeded: rows [len, len+B) <- block rows, K and V.
