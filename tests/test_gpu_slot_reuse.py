@@ -10,7 +10,7 @@ from paper_2504_15364_b200 import KeyDiff, KeyDiffError, binding, synth
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-PATHS = [binding.KEYDIFF_PATH_STAGED]
+PATHS = [binding.KEYDIFF_PATH_STAGED, binding.KEYDIFF_PATH_FUSED]
 SLOTS = binding.KEYDIFF_COMPACT_SLOT_REUSE
 RAW = binding.KEYDIFF_ANCHOR_RAW_MEAN
 
