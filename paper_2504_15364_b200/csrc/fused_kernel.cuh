@@ -318,10 +318,11 @@ __device__ __forceinline__ int find_crossing(const int* h, int E, int lane, int 
 // copy and gets the same answer): 2048-bin histogram, exact rank inside the threshold bin, radix
 // select when that bin is crowded; then an ordered scan gives every kept row of this CTA's slice
 // its destination (evicted: -1 - the number of evicted tokens before it), misc[1] the index of the first
-// evicted token and misc[4] the number of evicted tokens among the first `len`.
+// evicted token and misc[4] the number of evicted tokens among the first `len`.  With evict_bitmap the
+// evicted tokens' bits are set there as well (pass seg_a = seg_b to skip the destinations).
 __device__ __noinline__ void full_select_plan(const uint32_t* keys, int n, int N, int seg_a, int seg_b, int* hist,
                                               uint32_t* cand_key, int* cand_idx, int* dst_of, SelectSmem& sel, int* misc,
-                                              int len) {
+                                              int len, uint32_t* evict_bitmap = nullptr) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;
     if (tid == 0) { misc[0] = 0; misc[1] = n; }
@@ -412,6 +413,7 @@ __device__ __noinline__ void full_select_plan(const uint32_t* keys, int n, int N
         const int kept_before = pre_gt + min(pre_eq, th.need_eq);
         if (i >= seg_a && i < seg_b) dst_of[i - seg_a] = keep ? kept_before : -1 - (i - kept_before);
         if (i == len) misc[4] = i - kept_before;
+        if (!keep && evict_bitmap) atomicOr(&evict_bitmap[i >> 5], 1u << (i & 31));   // (cleared by the caller)
         if (!keep) local_first = min(local_first, i);
         pre_gt += k > th.key;
         pre_eq += is_eq;

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "staged_kernels.cuh"
 #include "fused_kernel.cuh"
+#include "slot_kernel.cuh"
 
 namespace {
 
@@ -43,6 +44,9 @@ struct keydiff_ctx {
     int fused_smem_bytes = 0;
     int fused_max_clusters = 0; // co-resident clusters (grid = min(U, this) * cluster)
     int fused_reg_rows = 0;     // kernel instance: rows per row group kept in registers
+    bool slot_stream = false;   // slot reuse: the streaming kernel serves the step (cluster, fused_nkeys,
+    int slot_ring_tiles = 0;    //   fused_smem_bytes, fused_max_clusters describe it)
+    int slot_nwords = 0;
     // running anchor of the fused path: sum of k/||k|| over the cached rows, per unit
     bool incremental = true;    // use it (one-pass kernel) when it is valid
     bool anchor_valid = false;  // the buffers describe the cache as the last evicting step left it
@@ -111,8 +115,9 @@ FusedKernel fused_instance(int reg_rows, int* built, bool one_pass = false, bool
     return one_pass ? fused_instance_of<true, false>(reg_rows, built) : fused_instance_of<false, false>(reg_rows, built);
 }
 
-// Co-resident clusters of `C` CTAs of the fused kernel instance `kern` with `smem` bytes each.
-int max_active_clusters(FusedKernel kern, int C, int smem, int sm_count) {
+// Co-resident clusters of `C` CTAs of the kernel `kern` with `smem` bytes each.
+template <typename Kernel>
+int max_active_clusters(Kernel kern, int C, int smem, int sm_count) {
     using namespace kd;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return 0;
     if (C > 8 && cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return 0;
@@ -170,7 +175,93 @@ bool plan_fused(keydiff_ctx* c, int sm_count) {
            max_active_clusters(fused_instance(c->fused_reg_rows, &built, true, slot_reuse(c)), c->cluster, c->fused_smem_bytes, sm_count) >= 1;
 }
 
+// Slot reuse: cluster size and ring of the streaming kernel for units of up to nmax rows; false if it
+// cannot serve the configuration (then the resident kernel or the staged path does).  Nothing has to
+// stay on chip, so small clusters are possible and many units are in flight; the estimate
+//   ceil(U / clusters) * (fixed cost per unit + cost per slice row * slice rows)
+// picks the size (constants from per-phase timings on a B200: anchor, selection, lists and barriers are
+// a fixed cost, the stream runs at the pace of one SM's share of the HBM bandwidth).
+bool plan_slot_stream(keydiff_ctx* c, int sm_count) {
+    using namespace kd;
+    if (c->cfg.max_block > kSlotMaxBlock) return false;
+    int forced = 0;
+    if (const char* env = std::getenv("KEYDIFF_CLUSTER_SIZE")) forced = std::atoi(env);   // tuning aid
+    const int nwords = (c->nmax + 31) / 32;
+    double best = 0.0;
+    bool found = false;
+    for (int C = 1; C <= kMaxCluster; ++C) {
+        if (forced > 0 && C != forced) continue;
+        const int per_cta = ((c->nmax + C - 1) / C + kTileRows - 1) / kTileRows * kTileRows;
+        const int nkeys = C * per_cta;
+        int ring = 3 * kFusedWarps;   // up to three tiles per warp in flight
+        while (ring > 0 && slot_layout(ring, nkeys, nwords, c->cfg.max_block).total > kSmemLimit) ring -= kFusedWarps;
+        if (ring <= 0) continue;
+        const int smem = slot_layout(ring, nkeys, nwords, c->cfg.max_block).total;
+        const int clusters = max_active_clusters(slot_evict_kernel, C, smem, sm_count);
+        if (clusters < 1) continue;
+        const int used = std::min(c->U, clusters);
+        const double row_us = 256.0 / (6.0e6 / std::min(sm_count, used * C));   // one SM's share of ~6 TB/s, in bytes per us
+        const double est = static_cast<double>((c->U + used - 1) / used) * ((C > 1 ? 11.0 : 9.0) + std::max(row_us, 0.0045) * per_cta);
+        if (!found || est < best) {
+            found = true; best = est;
+            c->cluster = C; c->fused_nkeys = nkeys; c->fused_smem_bytes = smem; c->fused_max_clusters = clusters;
+            c->slot_ring_tiles = ring; c->slot_nwords = nwords;
+        }
+    }
+    if (!found) return false;
+    return max_active_clusters(slot_evict_kernel, c->cluster, c->fused_smem_bytes, sm_count) >= 1;
+}
+
+int launch_slot_stream(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const uint4* nv, int B, cudaStream_t st) {
+    using namespace kd;
+    const int N = c->cfg.budget, n = c->len + B;
+    if (!(c->incremental && c->anchor_valid && c->steps_since_full < 1024)) {
+        // the running sum of the cached rows, rebuilt from all of them: first evicting step, after appends,
+        // set_len / reset, periodically against rounding drift, and every step when the caller asked for it
+        const int rows_per_split = (c->len + c->splits - 1) / c->splits;
+        anchor_partial_kernel<<<dim3(c->splits, c->U), kStagedThreads, 0, st>>>(kc, nk, c->len, 0, N, c->eps, rows_per_split, c->nmax,
+                                                                               c->partial, c->norms, c->cfg.anchor_mode == KEYDIFF_ANCHOR_RAW_MEAN);
+        anchor_fold_kernel<<<c->U, kHeadDim, 0, st>>>(c->partial, c->splits, c->anchor_sum[c->anchor_par], c->anchor_delta, c->cluster);
+        c->steps_since_full = 0;
+    } else {
+        ++c->steps_since_full;
+    }
+    SlotParams p;
+    p.k_cache = kc; p.v_cache = vc; p.new_k = nk; p.new_v = nv;
+    p.len = c->len; p.B = B; p.N = N; p.U = c->U; p.eps = c->eps;
+    p.cluster = c->cluster;
+    p.rows_per_cta = ((n + c->cluster - 1) / c->cluster + kTileRows - 1) / kTileRows * kTileRows;
+    p.ring_tiles = c->slot_ring_tiles; p.nkeys = c->fused_nkeys; p.nwords = c->slot_nwords; p.nmax = c->nmax;
+    p.max_block = c->cfg.max_block;
+    p.scores = c->scores; p.kept_idx = c->kept_idx; p.first_evicted = c->first_evicted;
+    p.moved_rows = c->moved_rows; p.status = c->status;
+    p.anchor_in = c->anchor_sum[c->anchor_par];
+    p.anchor_out = c->anchor_sum[c->anchor_par ^ 1];
+    p.anchor_delta = c->anchor_delta;
+    p.raw_anchor = c->cfg.anchor_mode == KEYDIFF_ANCHOR_RAW_MEAN;
+    p.window = c->cfg.recent_window;
+    p.pos = c->pos; p.next_pos = static_cast<int>(c->next_pos);
+    const int nclusters = std::min(c->U, c->fused_max_clusters);
+    p.stagger_ns = 0;
+    if (const char* env = std::getenv("KEYDIFF_STAGGER_NS")) p.stagger_ns = static_cast<unsigned>(std::atoi(env));   // tuning aid
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(nclusters * c->cluster);
+    cfg.blockDim = dim3(kFusedThreads);
+    cfg.dynamicSmemBytes = c->fused_smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = c->cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    KD_CUDA(cudaLaunchKernelEx(&cfg, slot_evict_kernel, p));
+    KD_CUDA(cudaGetLastError());
+    c->anchor_par ^= 1;
+    c->anchor_valid = true;
+    return KEYDIFF_OK;
+}
+
 int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const uint4* nv, int B, cudaStream_t st) {
+    if (c->slot_stream) return launch_slot_stream(c, kc, vc, nk, nv, B, st);
     using namespace kd;
     FusedParams p;
     p.k_cache = kc; p.v_cache = vc; p.new_k = nk; p.new_v = nv;
@@ -309,7 +400,9 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
     }
     if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
     if (ok && cfg->path != KEYDIFF_PATH_STAGED) {
-        if (plan_fused(c, prop.multiProcessorCount)) {
+        const bool use_stream = slot_reuse(c) && !std::getenv("KEYDIFF_SLOT_RESIDENT") && plan_slot_stream(c, prop.multiProcessorCount);
+        c->slot_stream = use_stream;
+        if (use_stream || plan_fused(c, prop.multiProcessorCount)) {
             c->path = KEYDIFF_PATH_FUSED;
             const size_t sum_bytes = sizeof(double) * U * kd::kHeadDim;
             ok = cudaMalloc(&c->anchor_sum[0], sum_bytes) == cudaSuccess && cudaMalloc(&c->anchor_sum[1], sum_bytes) == cudaSuccess &&

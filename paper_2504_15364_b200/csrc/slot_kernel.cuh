@@ -1,0 +1,470 @@
+// The eviction step with unordered slot reuse as one streaming kernel.
+//
+// Eq. (keydiff) gathers the kept rows, K' = gather(K, S), without fixing their order, and attention does
+// not depend on the order of the cached pairs.  With slot reuse the kept cache rows stay where they are
+// and the kept block rows are written into the freed slots, so the step only has to READ the unit's keys
+// once (to score them, App. B.1) and to write at most B rows of K and V.  Nothing has to stay on chip:
+// a cluster of C CTAs (C may be 1) streams its unit's K rows through a ring of 16-row tiles in shared
+// memory, warp w owning ring slots w, w+16, ...: it waits for a tile, scores its rows against the anchor
+// (known beforehand from the running sum, see fused_kernel.cuh), and at once refills the slot with the
+// next tile of its stream, which runs on into the cluster's next unit.  The loads of a unit therefore
+// arrive while the previous unit is being selected.
+//
+//   anchor   running sum + deltas + the block rows' terms (every CTA normalises the whole block)
+//   scores   per tile as it lands; keys into the CTA's table; the slice's keys pushed to the peers (DSMEM)
+//   select   every CTA on its own full copy of the table (the low-end select of fused_kernel.cuh, or the
+//            full-table select); result: the bitmap of evicted candidates, the same in every CTA
+//   place    from the bitmap every CTA derives the same three lists (evicted candidates, freed slots,
+//            kept block rows); row group number r of the cluster reads evicted row r once more (its
+//            k/||k|| leaves the running sum) and writes kept block row r into freed slot r
+//
+// One cluster barrier per unit (all keys delivered) plus a split one that keeps a peer's next push away
+// from a table still being read; none when C = 1.  Every wait is bounded (status word on expiry).
+#pragma once
+#include "fused_kernel.cuh"
+
+namespace kd {
+
+constexpr int kSlotMaxBlock = 1024;   // the three lists of a step live in shared memory, max_block entries each
+
+struct SlotLayout {
+    int ring, keys, work, bitmap, cand, lists, sel, mu, mbar, misc, total;
+};
+__host__ __device__ inline SlotLayout slot_layout(int ring_tiles, int nkeys, int nwords, int max_block) {
+    SlotLayout L;
+    int off = 0;
+    auto take = [&off](int bytes) { const int o = off; off += (bytes + 127) & ~127; return o; };
+    L.ring = take(ring_tiles * kTileRows * kRowBytes);
+    L.keys = take(nkeys * 4 > kBins * 4 ? nkeys * 4 : kBins * 4);   // also 8 KB of reduction scratch while the table is dead
+    L.work = take(kBins * 4);            // warp-reduction scratch / histogram
+    L.bitmap = take(2 * nwords * 4);     // evicted-candidate bitmap, evicted-before count of every word
+    L.cand = take(2 * kCandCap * 4);     // keys and indices of the threshold bin
+    L.lists = take(3 * max_block * 4);   // evicted candidates, freed slots, kept block rows
+    L.sel = take(static_cast<int>(sizeof(SelectSmem)));
+    L.mu = take(kHeadDim * 4);
+    L.mbar = take(ring_tiles * 8);
+    L.misc = take(128);
+    L.total = off;
+    return L;
+}
+
+struct SlotParams {
+    uint4* k_cache; uint4* v_cache; const uint4* new_k; const uint4* new_v;
+    int len, B, N, U;
+    float eps;
+    int cluster;        // CTAs per cluster
+    int rows_per_cta;   // slice length, a multiple of kTileRows
+    int ring_tiles;     // tiles in the ring, a multiple of the warp count
+    int nkeys;          // key-table capacity (>= cluster * rows_per_cta)
+    int nwords;         // bitmap words provided for (>= ceil(n / 32))
+    int nmax;           // row stride of the score scratch
+    int max_block;
+    unsigned stagger_ns;
+    float* scores; int32_t* kept_idx; int32_t* first_evicted;
+    unsigned long long* moved_rows; int32_t* status;
+    const double* anchor_in; double* anchor_out; float* anchor_delta;   // running anchor, as in FusedParams
+    int raw_anchor, window;
+    int32_t* pos;       // [U][N] token position of every slot
+    int next_pos;       // position of the block's first token
+};
+
+// One thread: bulk-load unit rows [g0, g0 + nrows) of unit u (cache rows below len, block rows after) to dst.
+__device__ __forceinline__ void issue_rows(const uint4* cache, const uint4* block, int u, int len, int B, int N,
+                                           int g0, int nrows, uint32_t dst, uint32_t bar) {
+    const int from_cache = min(max(len - g0, 0), nrows);
+    const int from_block = nrows - from_cache;
+    mbar_expect_tx(bar, nrows * kRowBytes);
+    if (from_cache > 0)
+        bulk_load(dst, cache + (static_cast<size_t>(u) * N + g0) * kRowVec, from_cache * kRowBytes, bar);
+    if (from_block > 0)
+        bulk_load(dst + from_cache * kRowBytes,
+                  block + (static_cast<size_t>(u) * B + (g0 + from_cache - len)) * kRowVec, from_block * kRowBytes, bar);
+}
+
+__global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const SlotParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int C = p.cluster;
+    const SlotLayout L = slot_layout(p.ring_tiles, p.nkeys, p.nwords, p.max_block);
+    const uint4* ring = reinterpret_cast<const uint4*>(smem + L.ring);
+    uint32_t* keys = reinterpret_cast<uint32_t*>(smem + L.keys);
+    int* hist = reinterpret_cast<int*>(smem + L.work);
+    float* red = reinterpret_cast<float*>(smem + L.work);
+    uint32_t* bitmap = reinterpret_cast<uint32_t*>(smem + L.bitmap);
+    int* wlocal = reinterpret_cast<int*>(smem + L.bitmap) + p.nwords;
+    uint32_t* cand_key = reinterpret_cast<uint32_t*>(smem + L.cand);
+    int* cand_idx = reinterpret_cast<int*>(smem + L.cand) + kCandCap;
+    int* ev_of = reinterpret_cast<int*>(smem + L.lists);   // evicted candidates, ascending
+    int* slot_of = ev_of + p.max_block;                    // freed slots, ascending
+    int* blk_of = slot_of + p.max_block;                   // kept block rows, ascending
+    SelectSmem& sel = *reinterpret_cast<SelectSmem*>(smem + L.sel);
+    float* mu_sh = reinterpret_cast<float*>(smem + L.mu);
+    int* misc = reinterpret_cast<int*>(smem + L.misc);   // 0 ncand, 1 first evicted, 2 need_eq, 3 threshold key, 4 evicted cache rows
+    const uint32_t ring_sa = smem_addr(ring), mbar_sa = smem_addr(smem + L.mbar), keys_sa = smem_addr(keys);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = tid >> 3, t = tid & 7, sub = lane >> 3;
+    const int crank = static_cast<int>(cluster_ctarank());
+    const int cluster_id = blockIdx.x / C, nclusters = gridDim.x / C;
+    const int len = p.len, B = p.B, N = p.N, n = len + B, E = n - N;   // E candidates are evicted
+    const float inv_eps = 1.0f / p.eps;
+    const bool raw = p.raw_anchor != 0;
+    const int nwords = (n + 31) >> 5;
+    const bool fast_ok = n <= kFastKeys * kFusedThreads && nwords <= kFusedThreads;
+    const int seg_a = min(n, crank * p.rows_per_cta);
+    const int seg = min(n, seg_a + p.rows_per_cta) - seg_a, seg_b = seg_a + seg;
+    // The slice as a stream of 16-row tiles; warp w takes tiles w, w+16, ... of every unit of the cluster,
+    // one unit after the other, through its own D ring slots (slot w + 16 d).
+    const int nvt = (seg + kTileRows - 1) / kTileRows;
+    const int cnt_w = warp < nvt ? (nvt - warp + kFusedWarps - 1) / kFusedWarps : 0;   // tiles per unit for this warp
+    const int D = p.ring_tiles / kFusedWarps;
+    const int my_units = cluster_id < p.U ? (p.U - cluster_id + nclusters - 1) / nclusters : 0;
+
+    if (tid == 0) {
+        for (int j = 0; j < p.ring_tiles; ++j) mbar_init(mbar_sa + 8 * j, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (p.stagger_ns != 0 && cluster_id != 0) {   // bounded start-up delay that spreads the clusters' phases
+        const unsigned long long t0 = global_timer_ns();
+        const unsigned long long wait_ns = static_cast<unsigned long long>(p.stagger_ns) * static_cast<unsigned>(cluster_id);
+        for (int spin = 0; spin < (1 << 16) && global_timer_ns() - t0 < wait_ns; ++spin) __nanosleep(100);
+    }
+
+    // issue side of the warp's stream: the next tile to request is tile i_j of the cluster's i_it-th unit
+    int i_it = 0, i_j = 0;
+    auto issue_next = [&](int d) {   // lane 0 only; d = ring slot (of this warp) to fill
+        const int vt = warp + kFusedWarps * i_j;
+        const int lo = vt * kTileRows, hi = min(seg, lo + kTileRows);
+        const int phys = warp + kFusedWarps * d;
+        issue_rows(p.k_cache, p.new_k, cluster_id + i_it * nclusters, len, B, N, seg_a + lo, hi - lo,
+                   ring_sa + phys * kTileRows * kRowBytes, mbar_sa + 8 * phys);
+        if (++i_j == cnt_w) { i_j = 0; ++i_it; }
+    };
+    if (lane == 0 && cnt_w > 0)
+        for (int d = 0; d < D && i_it < my_units; ++d) issue_next(d);
+    int c_d = 0;            // ring slot the next tile of the stream arrives in
+    uint32_t c_par = 0;     // bit d: parity the next wait on slot d expects
+    bool exchange_pending = false;   // an arrive of the split cluster barrier has no wait yet
+
+    for (int u = cluster_id; u < p.U; u += nclusters) {
+        const int un = u + nclusters;
+        float block_sum = 0.f;   // tid < 128: channel tid of the block rows' sum of k/||k||
+        // ------------------------------------------------------------ anchor from the running sum + the block rows
+        {
+            double run = 0.0;
+            float dl[kMaxCluster];
+            if (tid < kHeadDim) {
+                run = p.anchor_in[static_cast<size_t>(u) * kHeadDim + tid];
+#pragma unroll
+                for (int c = 0; c < kMaxCluster; ++c)
+                    dl[c] = c < C ? p.anchor_delta[(static_cast<size_t>(u) * C + c) * kHeadDim + tid] : 0.f;
+            }
+            float2 acc[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc[q] = make_float2(0.f, 0.f);
+            for (int b0 = 0; b0 < B; b0 += kGroups) {   // (same trip count in every lane: row_a1 shuffles)
+                const int br = b0 + g;
+                uint4 a = make_uint4(0, 0, 0, 0), b = a;
+                if (br < B) {
+                    const uint4* row = p.new_k + (static_cast<size_t>(u) * B + br) * kRowVec;
+                    a = row[t]; b = row[t + 8];
+                }
+                row_a1(a, b, br < B, inv_eps, acc, raw);
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                float2 v = acc[q];
+                v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
+                v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
+                acc[q] = v;
+            }
+            if (lane < 8) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<float2*>(&red[warp * kHeadDim + lane_channel(t, 2 * q)]) = acc[q];
+            }
+            __syncthreads();
+            if (tid < kHeadDim) {
+#pragma unroll
+                for (int w = 0; w < kFusedWarps; ++w) block_sum += red[w * kHeadDim + tid];
+                double a = run;
+#pragma unroll
+                for (int c = 0; c < kMaxCluster; ++c) a += static_cast<double>(dl[c]);   // rank order; absent ranks add 0
+                if (crank == 0) p.anchor_out[static_cast<size_t>(u) * kHeadDim + tid] = a;   // the cached rows' sum, folded
+                mu_sh[tid] = static_cast<float>((a + static_cast<double>(block_sum)) / static_cast<double>(n));
+            }
+            __syncthreads();
+        }
+        // ------------------------------------------------------------ a1 + a2 in one pass over the stream
+        {
+            float2 w[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) w[q] = *reinterpret_cast<const float2*>(&mu_sh[lane_channel(t, 2 * q)]);
+            float m;   // ||mu||, computed by every warp in the same order
+            {
+                const float4 c4 = reinterpret_cast<const float4*>(mu_sh)[lane];
+                float v = fmaf(c4.w, c4.w, fmaf(c4.z, c4.z, fmaf(c4.y, c4.y, c4.x * c4.x)));
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                m = sqrtf(v);
+            }
+#pragma unroll 1
+            for (int j = 0; j < cnt_w; ++j) {
+                const int phys = warp + kFusedWarps * c_d;
+                mbar_wait(mbar_sa + 8 * phys, (c_par >> c_d) & 1u, p.status);
+                c_par ^= 1u << c_d;
+                const int lo = (warp + kFusedWarps * j) * kTileRows;   // first slice row of the tile
+                const uint4* tile = ring + phys * kTileRows * kRowVec;
+                float v[8];   // this lane's shares of the tile's four rows of its row group
+#pragma unroll
+                for (int it = 0; it < 4; ++it) {
+                    const int r = it * 4 + sub;
+                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
+                    if (lo + r < seg) { a = tile[r * kRowVec + t]; b = tile[r * kRowVec + t + 8]; }
+                    lane_sumsq_dot(a, b, w, v[2 * it], v[2 * it + 1]);
+                }
+                const uint32_t key = score4(v, t, m, p.eps);
+                const int lr = lo + (t >> 1) * 4 + sub;
+                if (!(t & 1) && lr < seg) keys[seg_a + lr] = key;
+                __syncwarp();   // the tile's only readers are this warp's lanes: the copy engine may refill it
+                if (lane == 0 && i_it < my_units) issue_next(c_d);
+                if (++c_d == D) c_d = 0;
+            }
+        }
+        if (exchange_pending) { cluster_wait(); exchange_pending = false; }   // the peers are done with the previous unit's table
+        __syncthreads();
+        if (C > 1) {
+            // this slice's keys -> every peer's table (128-bit DSMEM stores; slices are multiples of 16 rows)
+            const uint4* mine = reinterpret_cast<const uint4*>(keys + seg_a);
+            for (int c = 1; c < C; ++c) {
+                const int peer = crank + c < C ? crank + c : crank + c - C;
+                const uint32_t base = map_to_cta(keys_sa + 4 * seg_a, peer);
+                for (int o = tid; 4 * o < seg; o += kFusedThreads) st_cluster_v4(base + 16 * o, mine[o]);
+            }
+            cluster_arrive();
+        }
+        {
+            float* sc = p.scores + static_cast<size_t>(u) * p.nmax + seg_a;   // fp32 scores to global scratch, coalesced
+            for (int lr = tid; lr < seg; lr += kFusedThreads) sc[lr] = key_score(keys[seg_a + lr]);
+            for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;
+            for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;
+            if (tid == 0) { misc[0] = 0; misc[1] = n; }
+        }
+        if (C > 1) cluster_wait();   // (2) the key table of every CTA holds all n keys
+        __syncthreads();
+        if (p.window > 0) {
+            // sliding window (Sec. 3.2): tokens at the last `window` positions of the sequence get the largest
+            // possible key, so they are never among the E smallest
+            const int first_recent = p.next_pos + B - p.window;
+            for (int i = len + max(B - p.window, 0) + tid; i < n; i += kFusedThreads) keys[i] = 0xffffffffu;
+            if (p.window > B) {
+                const int32_t* ps = p.pos + static_cast<size_t>(u) * N;
+                for (int i = tid; i < len; i += kFusedThreads) if (ps[i] >= first_recent) keys[i] = 0xffffffffu;
+            }
+            __syncthreads();
+        }
+        // ------------------------------------------------------------ a3: the bitmap of evicted candidates
+        bool planned = false;
+        int* wbase = sel.hist + 2 * kFusedWarps;
+        if (fast_ok) {
+            // the low-end select of fused_kernel.cuh: keys in registers, 2048 bins over the low end of the unit's
+            // own key range, candidates under the threshold bin straight into the bitmap, the bin's own keys
+            // ranked exactly under (key ascending, candidate number descending)
+            uint32_t* wmin = reinterpret_cast<uint32_t*>(sel.hist);
+            uint32_t* wmax = reinterpret_cast<uint32_t*>(sel.hist) + kFusedWarps;
+            const int cnt = (n - tid + kFusedThreads - 1) / kFusedThreads;
+            uint32_t kk[kFastKeys];
+#pragma unroll
+            for (int j = 0; j < kFastKeys; ++j) kk[j] = j < cnt ? keys[tid + j * kFusedThreads] : 0xffffffffu;
+            {
+                uint32_t lo = 0xffffffffu, hi = 0u;
+#pragma unroll
+                for (int j = 0; j < kFastKeys; ++j) { lo = min(lo, kk[j]); if (j < cnt) hi = max(hi, kk[j]); }
+                const uint32_t cut = (n >= kFusedThreads && E <= kFusedThreads) ? lo : hi;   // bounds the E-th smallest key
+                const uint32_t wlo = __reduce_min_sync(0xffffffffu, lo);
+                const uint32_t wcut = __reduce_max_sync(0xffffffffu, cnt > 0 ? cut : 0u);
+                if (lane == 0) { wmin[warp] = wlo; wmax[warp] = wcut; }
+            }
+            __syncthreads();
+            uint32_t kmin, kcut, shift;
+            {
+                const uint32_t lo = lane < kFusedWarps ? wmin[lane] : 0xffffffffu, hi = lane < kFusedWarps ? wmax[lane] : 0u;
+                kmin = __reduce_min_sync(0xffffffffu, lo);
+                kcut = __reduce_max_sync(0xffffffffu, hi);
+                const int bits = 32 - __clz(kcut - kmin);
+                shift = bits > 11 ? bits - 11 : 0;
+            }
+            auto bin_of = [kmin, kcut, shift](uint32_t k) { return k <= kcut ? min((k - kmin) >> shift, 2046u) : 2047u; };
+#pragma unroll
+            for (int j = 0; j < kFastKeys; ++j) if (j < cnt) atomicAdd(&hist[bin_of(kk[j])], 1);
+            __syncthreads();
+            const int packed = find_crossing(hist, E, lane, warp, sel.warp_eq);
+            const uint32_t bstar = static_cast<uint32_t>(packed >> 16);
+            const int need = E - (packed & 0xffff);   // this many keys of the threshold bin go
+            unsigned m_below = 0, m_in = 0;
+#pragma unroll
+            for (int j = 0; j < kFastKeys; ++j) {
+                const uint32_t b = bin_of(kk[j]);
+                m_below |= (j < cnt && b < bstar) ? 1u << j : 0u;
+                m_in |= (j < cnt && b == bstar) ? 1u << j : 0u;
+            }
+            if (packed >= 0 && (m_below | m_in)) {
+                int first = n;
+                for (unsigned mm = m_below; mm; mm &= mm - 1) {
+                    const int i = tid + (__ffs(mm) - 1) * kFusedThreads;
+                    atomicOr(&bitmap[i >> 5], 1u << (i & 31));
+                    first = min(first, i);
+                }
+                for (unsigned mm = m_in; mm; mm &= mm - 1) {
+                    const int i = tid + (__ffs(mm) - 1) * kFusedThreads;
+                    const int slot = atomicAdd(&misc[0], 1);
+                    if (slot < kFastCandCap) { cand_key[slot] = keys[i]; cand_idx[slot] = i; }
+                }
+                if (first < n) atomicMin(&misc[1], first);
+            }
+            __syncthreads();
+            const int ncand = misc[0];
+            if (packed >= 0 && ncand <= kFastCandCap) {   // uniform: every thread sees the same values
+                int wfirst = n;
+                for (int c = warp; c < ncand; c += kFusedWarps) {
+                    const uint32_t mk = cand_key[c];
+                    const int mi = cand_idx[c];
+                    int rank = 0;
+                    for (int q = lane; q < ncand; q += 32) {
+                        const uint32_t ok = cand_key[q];
+                        rank += (ok < mk) || (ok == mk && cand_idx[q] > mi);
+                    }
+                    rank = __reduce_add_sync(0xffffffffu, rank);
+                    if (lane == 0 && rank < need) { atomicOr(&bitmap[mi >> 5], 1u << (mi & 31)); wfirst = min(wfirst, mi); }
+                }
+                if (lane == 0 && wfirst < n) atomicMin(&misc[1], wfirst);
+                planned = true;
+            }
+            __syncthreads();
+        }
+        if (!planned) {
+            // the full-table select writes the same bitmap (cleared first: the attempt above may have marked some)
+            for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;
+            __syncthreads();
+            full_select_plan(keys, n, N, 0, 0, hist, cand_key, cand_idx, nullptr, sel, misc, len, bitmap);
+        }
+        {
+            // evicted candidates before each word of the bitmap
+            for (int w0 = 0; w0 < nwords; w0 += kFusedThreads) {   // (nwords <= 512 on the low-end route; any size here)
+                const int wi = w0 + tid;
+                const int pc = wi < nwords ? __popc(bitmap[wi]) : 0;
+                int incl = pc;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += v;
+                }
+                if (wi < nwords) wlocal[wi] = incl - pc;   // within its warp's 32 words
+                if (lane == 31) sel.warp_gt[warp] = incl;
+                __syncthreads();
+                if (warp == 0) {
+                    const int t2 = lane < kFusedWarps ? sel.warp_gt[lane] : 0;
+                    int incl2 = t2;
+#pragma unroll
+                    for (int o = 1; o < 16; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl2, o); if (lane >= o) incl2 += v; }
+                    if (lane < kFusedWarps) wbase[lane] = incl2 - t2 + (w0 > 0 ? misc[5] : 0);
+                    if (lane == kFusedWarps - 1) misc[6] = incl2 + (w0 > 0 ? misc[5] : 0);
+                }
+                __syncthreads();
+                if (wi < nwords) wlocal[wi] += wbase[warp];   // evicted candidates before word wi
+                if (tid == 0) misc[5] = misc[6];
+                __syncthreads();
+            }
+        }
+        auto evicted_before = [&](int i) { const int w = i >> 5; return wlocal[w] + __popc(bitmap[w] & ((1u << (i & 31)) - 1u)); };
+        // ------------------------------------------------------------ the three lists, the same in every CTA
+        const int evicted_cache = evicted_before(len);   // evicted candidates among the len cache slots (len < n)
+        const int kept_cache = len - evicted_cache;
+        const int kb = N - kept_cache;                   // kept block rows = freed slots
+        for (int w = tid; w < nwords; w += kFusedThreads) {
+            int e = wlocal[w];
+            for (uint32_t wd = bitmap[w]; wd; wd &= wd - 1) {
+                const int i = 32 * w + __ffs(wd) - 1;
+                ev_of[e] = i;
+                if (i < len) slot_of[e] = i;   // every candidate before a cache slot is a cache slot
+                ++e;
+            }
+        }
+        for (int j = tid; j < B; j += kFusedThreads) {
+            const int i = len + j;
+            if (!((bitmap[i >> 5] >> (i & 31)) & 1u)) blk_of[(i - evicted_before(i)) - kept_cache] = j;
+        }
+        for (int e = len + tid; e < N; e += kFusedThreads) slot_of[evicted_cache + (e - len)] = e;   // slots that were still empty
+        // kept cache rows of this slice keep their slot: the kept-index list says so
+        for (int i = seg_a + tid; i < min(seg_b, len); i += kFusedThreads)
+            if (!((bitmap[i >> 5] >> (i & 31)) & 1u)) p.kept_idx[static_cast<size_t>(u) * N + i] = i;
+        if (crank == 0 && tid == 0) {
+            p.first_evicted[u] = misc[1];
+            atomicAdd(p.moved_rows, static_cast<unsigned long long>(kb));
+        }
+        if (crank == 0 && un < p.U) {   // the next unit's block rows towards L2: every CTA reads them first thing
+            const char* nb = reinterpret_cast<const char*>(p.new_k + static_cast<size_t>(un) * B * kRowVec);
+            for (int o = tid * 128; o < B * kRowBytes; o += kFusedThreads * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(nb + o));
+        }
+        __syncthreads();
+        // ------------------------------------------------------------ a4: evicted rows leave the running sum, kept block rows take the freed slots
+        {
+            float2 gone[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) gone[q] = make_float2(0.f, 0.f);
+            const int todo = max(E, kb);
+            for (int r0 = 0; r0 < todo; r0 += C * kGroups) {   // (same trip count in every lane: row_a1 shuffles)
+                const int r = r0 + crank * kGroups + g;
+                const bool ev = r < E;
+                if (__any_sync(0xffffffffu, ev)) {
+                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
+                    if (ev) {
+                        const uint4* row = concat_row(p.k_cache, p.new_k, u, ev_of[r], len, B, N);
+                        a = row[t]; b = row[t + 8];
+                    }
+                    row_a1(a, b, ev, inv_eps, gone, raw);
+                }
+                if (r < kb) {
+                    // freed slot r is evicted cache row r for r < evicted_cache: the lanes that read its old words
+                    // above are the ones that overwrite them here
+                    const int slot = slot_of[r], j = blk_of[r];
+                    const uint4* sk = p.new_k + (static_cast<size_t>(u) * B + j) * kRowVec;
+                    const uint4* sv = p.new_v + (static_cast<size_t>(u) * B + j) * kRowVec;
+                    uint4* dk = p.k_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
+                    uint4* dv = p.v_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
+                    dk[t] = sk[t]; dk[t + 8] = sk[t + 8];
+                    dv[t] = sv[t]; dv[t + 8] = sv[t + 8];
+                    if (t == 0) {
+                        p.kept_idx[static_cast<size_t>(u) * N + slot] = len + j;
+                        p.pos[static_cast<size_t>(u) * N + slot] = p.next_pos + j;
+                    }
+                }
+            }
+            float* red2 = reinterpret_cast<float*>(keys);   // the key table is dead until the next unit
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                float2 v = gone[q];
+                v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
+                v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
+                gone[q] = v;
+            }
+            if (lane < 8) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<float2*>(&red2[warp * kHeadDim + lane_channel(t, 2 * q)]) = gone[q];
+            }
+            __syncthreads();
+            if (tid < kHeadDim) {
+                float e = 0.f;
+#pragma unroll
+                for (int w = 0; w < kFusedWarps; ++w) e += red2[w * kHeadDim + tid];
+                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (crank == 0 ? block_sum : 0.f) - e;
+            }
+        }
+        if (C > 1) { cluster_arrive(); exchange_pending = true; }   // this CTA is done with the unit's key table
+        __syncthreads();   // the scratch areas are free for the next unit
+    }
+    if (exchange_pending) cluster_wait();
+    if (C > 1) cluster_sync_all();   // no CTA leaves while a peer may still address its shared memory
+}
+
+}  // namespace kd

@@ -237,6 +237,17 @@ slot_place_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
     if (tid == 0) atomicAdd(moved_rows, static_cast<unsigned long long>(kb));
 }
 
+// Running anchor of the cached rows from the partial sums of anchor_partial_kernel run over the cache
+// alone: sum[u][c] = sum over splits (double), and the pending deltas are cleared.  grid = U, 128 threads.
+__global__ void anchor_fold_kernel(const float* __restrict__ partial, int splits, double* __restrict__ sum,
+                                   float* __restrict__ delta, int ranks) {
+    const int u = blockIdx.x, c = threadIdx.x;
+    double a = 0.0;
+    for (int s = 0; s < splits; ++s) a += static_cast<double>(partial[(static_cast<size_t>(u) * splits + s) * kHeadDim + c]);
+    sum[static_cast<size_t>(u) * kHeadDim + c] = a;
+    for (int r = 0; r < ranks; ++r) delta[(static_cast<size_t>(u) * ranks + r) * kHeadDim + c] = 0.f;
+}
+
 // Token positions of the slots: identity (a cache the caller filled in token order) ...
 __global__ void pos_iota_kernel(int32_t* __restrict__ pos, int N, int total) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
