@@ -96,13 +96,6 @@ struct FusedParams {
     const double* anchor_in; double* anchor_out; float* anchor_delta;
     int raw_anchor;     // 1: the anchor is the mean of the keys themselves (Sec. 3.2), 0: of the normalised keys
     int window;         // w most recent tokens that are never evicted (Sec. 3.2, sliding window)
-    // unordered slot reuse (kSlots instances): token position of every slot, position of the block's first
-    // token, and two per-unit lists the CTAs of a cluster hand to one another through global memory
-    int32_t* pos;       // [U][N]
-    int next_pos;
-    int32_t* slot_of;   // [U][max_block]: the r-th freed slot
-    int32_t* blk_of;    // [U][max_block]: the r-th kept block row
-    int max_block;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -317,12 +310,12 @@ __device__ __forceinline__ int find_crossing(const int* h, int E, int lane, int 
 // Exact top-N over the whole key table by one CTA (every CTA of the cluster runs it on its own
 // copy and gets the same answer): 2048-bin histogram, exact rank inside the threshold bin, radix
 // select when that bin is crowded; then an ordered scan gives every kept row of this CTA's slice
-// its destination (evicted: -1 - the number of evicted tokens before it), misc[1] the index of the first
-// evicted token and misc[4] the number of evicted tokens among the first `len`.  With evict_bitmap the
-// evicted tokens' bits are set there as well (pass seg_a = seg_b to skip the destinations).
+// its destination (-1 = evicted) and misc[1] the index of the first evicted token.  With evict_bitmap the
+// evicted tokens' bits are set there as well (cleared by the caller; pass seg_a = seg_b to skip the
+// destinations).
 __device__ __noinline__ void full_select_plan(const uint32_t* keys, int n, int N, int seg_a, int seg_b, int* hist,
                                               uint32_t* cand_key, int* cand_idx, int* dst_of, SelectSmem& sel, int* misc,
-                                              int len, uint32_t* evict_bitmap = nullptr) {
+                                              uint32_t* evict_bitmap = nullptr) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;
     if (tid == 0) { misc[0] = 0; misc[1] = n; }
@@ -410,10 +403,8 @@ __device__ __noinline__ void full_select_plan(const uint32_t* keys, int n, int N
         const uint32_t k = keys[i];
         const bool is_eq = k == th.key;
         const bool keep = k > th.key || (is_eq && pre_eq < th.need_eq);
-        const int kept_before = pre_gt + min(pre_eq, th.need_eq);
-        if (i >= seg_a && i < seg_b) dst_of[i - seg_a] = keep ? kept_before : -1 - (i - kept_before);
-        if (i == len) misc[4] = i - kept_before;
-        if (!keep && evict_bitmap) atomicOr(&evict_bitmap[i >> 5], 1u << (i & 31));   // (cleared by the caller)
+        if (i >= seg_a && i < seg_b) dst_of[i - seg_a] = keep ? pre_gt + min(pre_eq, th.need_eq) : -1;
+        if (!keep && evict_bitmap) atomicOr(&evict_bitmap[i >> 5], 1u << (i & 31));
         if (!keep) local_first = min(local_first, i);
         pre_gt += k > th.key;
         pre_eq += is_eq;
@@ -434,12 +425,7 @@ __device__ __noinline__ void full_select_plan(const uint32_t* keys, int n, int N
 // anchor_delta, and the next step folds the deltas into the running sum in double precision, in a
 // fixed order.  kOnePass = false recomputes the anchor from all n rows (first evicting step, after
 // set_len / reset / appends, and periodically to shed rounding drift).
-//
-// kSlots: unordered slot reuse.  Eq. (keydiff) gathers the kept rows without fixing their order, so kept
-// cache rows can stay where they are: the unit's K rows are only read (scored), the next unit's K rows
-// start to arrive as soon as this unit's are scored, and after the selection the kept block rows are
-// written into the freed slots; V is touched for those rows only.
-template <int kRegRows, bool kOnePass, bool kSlots = false>
+template <int kRegRows, bool kOnePass>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const FusedParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int C = p.cluster;
@@ -715,26 +701,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             }
         }
         }   // kOnePass
-        if constexpr (kSlots) {
-            // the rows are not needed again: the next unit's K rows arrive under this unit's selection
-            if (un < p.U) {
-#pragma unroll 1
-                for (int s = 0; s < kTilesPerWarp; ++s) {
-                    const int tile = warp + kFusedWarps * s;
-                    if (tile >= ntiles) break;
-                    __syncwarp();   // the tile's only readers are this warp's lanes
-                    if (lane == 0) issue_tile(p.k_cache, p.new_k, un, len, B, N, sl, tile, rows_sa, mbar_sa);
-                }
-#pragma unroll
-                for (int k = 0; k < kRegRows; ++k) {
-                    const int lr = rs + k * kGroups + g;
-                    if (lr < seg) {
-                        const uint4* row = concat_row(p.k_cache, p.new_k, un, seg_a + lr, len, B, N);
-                        ra[k] = row[t]; rb[k] = row[t + 8];
-                    }
-                }
-            }
-        }
         __syncthreads();
         {
             // this slice's keys -> every peer's table (128-bit DSMEM stores)
@@ -760,17 +726,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             // sliding window (Sec. 3.2): the last `window` tokens get the largest possible key, so they are
             // never among the E smallest; the scores in global scratch stay what they are
             __syncthreads();   // this CTA's score write-out has read its keys
-            if constexpr (kSlots) {
-                // the cache is not in token order: "last" is read off the slots' token positions
-                const int first_recent = p.next_pos + B - p.window;
-                for (int i = len + max(B - p.window, 0) + tid; i < n; i += kFusedThreads) keys[i] = 0xffffffffu;
-                if (p.window > B) {
-                    const int32_t* ps = p.pos + static_cast<size_t>(u) * N;
-                    for (int i = tid; i < len; i += kFusedThreads) if (ps[i] >= first_recent) keys[i] = 0xffffffffu;
-                }
-            } else {
-                for (int i = n - p.window + tid; i < n; i += kFusedThreads) keys[i] = 0xffffffffu;
-            }
+            for (int i = n - p.window + tid; i < n; i += kFusedThreads) keys[i] = 0xffffffffu;
             __syncthreads();
         }
         // ------------------------------------------------------------ a3 + plan: who is evicted, where every kept row goes
@@ -880,105 +836,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 for (int lr = tid; lr < seg; lr += kFusedThreads) {
                     const int i = seg_a + lr, w = i >> 5;
                     const uint32_t wd = bitmap[w], bit = 1u << (i & 31);
-                    if constexpr (kSlots) {
-                        const int eb = wbase[w >> 5] + wlocal[w] + __popc(wd & (bit - 1));   // evicted tokens before i
-                        dst_of[lr] = (wd & bit) ? -1 - eb : i - eb;
-                    } else {
-                        dst_of[lr] = (wd & bit) ? -1 : i - (wbase[w >> 5] + wlocal[w] + __popc(wd & (bit - 1)));
-                    }
-                }
-                if constexpr (kSlots) {
-                    if (tid == 0) { const int w = len >> 5; misc[4] = wbase[w >> 5] + wlocal[w] + __popc(bitmap[w] & ((1u << (len & 31)) - 1u)); }
+                    dst_of[lr] = (wd & bit) ? -1 : i - (wbase[w >> 5] + wlocal[w] + __popc(wd & (bit - 1)));
                 }
                 __syncthreads();
                 planned = true;
             }
         }
-        if (!planned) full_select_plan(keys, n, N, seg_a, seg_b, hist, cand_key, cand_idx, dst_of, sel, misc, len);
-        if constexpr (kSlots) {
-        // ------------------------------------------------------------ a4 with slot reuse: kept block rows into the freed slots
-        const int evicted_cache = misc[4];            // evicted tokens among the len cache slots
-        const int kept_cache = len - evicted_cache;
-        const int kb = N - kept_cache;                // kept block rows = freed slots
-        int32_t* slot_of = p.slot_of + static_cast<size_t>(u) * p.max_block;
-        int32_t* blk_of = p.blk_of + static_cast<size_t>(u) * p.max_block;
-        if (crank == 0 && tid == 0) {
-            p.first_evicted[u] = misc[1];
-            atomicAdd(p.moved_rows, static_cast<unsigned long long>(kb));
-        }
-        // Each CTA knows, for the candidates of its slice, how many tokens before them are kept / evicted.
-        // Every token before a cache slot is a cache slot, so an evicted slot's count is its number among the
-        // freed slots; a kept block row's number among the kept block rows is its kept-before count minus the
-        // kept cache rows.  Both lists go to global scratch, where the whole cluster reads them.
-        for (int lr = tid; lr < seg; lr += kFusedThreads) {
-            const int i = seg_a + lr, d = dst_of[lr];
-            if (i < len) {
-                if (d >= 0) p.kept_idx[static_cast<size_t>(u) * N + i] = i;   // stays in its slot
-                else slot_of[-1 - d] = i;
-            } else if (d >= 0) {
-                blk_of[d - kept_cache] = i - len;
-            }
-        }
-        if (crank == 0)   // slots that were still empty come after the evicted ones
-            for (int e = len + tid; e < N; e += kFusedThreads) slot_of[evicted_cache + (e - len)] = e;
-        {
-            // what this CTA saw leave, for the running anchor: its evicted rows are read once more (from L2)
-            // before anybody may overwrite them
-            float2 gone[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) gone[q] = make_float2(0.f, 0.f);
-            if (kOnePass && crank == 0 && un < p.U) {   // the next unit's block rows towards L2: every CTA reads them first thing
-                const char* nb = reinterpret_cast<const char*>(p.new_k + static_cast<size_t>(un) * B * kRowVec);
-                for (int o = tid * 128; o < B * kRowBytes; o += kFusedThreads * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(nb + o));
-            }
-            for (int lr0 = 0; lr0 < seg; lr0 += kGroups) {   // (same trip count in every lane: row_a1 shuffles)
-                const int lr = lr0 + g;
-                const bool ev = lr < seg && dst_of[lr] < 0;
-                if (__any_sync(0xffffffffu, ev)) {
-                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
-                    if (ev) {
-                        const uint4* row = concat_row(p.k_cache, p.new_k, u, seg_a + lr, len, B, N);
-                        a = row[t]; b = row[t + 8];
-                    }
-                    row_a1(a, b, ev, inv_eps, gone, raw);
-                }
-            }
-            float* red2 = reinterpret_cast<float*>(keys);   // the key table is dead until the next unit
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                float2 v = gone[q];
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
-                gone[q] = v;
-            }
-            if (lane < 8) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    *reinterpret_cast<float2*>(&red2[warp * kHeadDim + lane_channel(t, 2 * q)]) = gone[q];
-            }
-            __syncthreads();
-            if (tid < kHeadDim) {
-                float e = 0.f;
-#pragma unroll
-                for (int w = 0; w < kFusedWarps; ++w) e += red2[w * kHeadDim + tid];
-                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass && crank == 0 ? block_sum : 0.f) - e;
-            }
-        }
-        cluster_sync_all();   // (3) both lists are complete; every CTA is done with its key table and exchange buffers
-        for (int r = crank * kGroups + g; r < kb; r += C * kGroups) {   // one row group per freed slot
-            const int slot = slot_of[r], j = blk_of[r];
-            const uint4* sk = p.new_k + (static_cast<size_t>(u) * B + j) * kRowVec;
-            const uint4* sv = p.new_v + (static_cast<size_t>(u) * B + j) * kRowVec;
-            uint4* dk = p.k_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
-            uint4* dv = p.v_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
-            dk[t] = sk[t]; dk[t + 8] = sk[t + 8];
-            dv[t] = sv[t]; dv[t + 8] = sv[t + 8];
-            if (t == 0) {
-                p.kept_idx[static_cast<size_t>(u) * N + slot] = len + j;
-                p.pos[static_cast<size_t>(u) * N + slot] = p.next_pos + j;
-            }
-        }
-        } else {
+        if (!planned) full_select_plan(keys, n, N, seg_a, seg_b, hist, cand_key, cand_idx, dst_of, sel, misc);
         const int first_evicted = misc[1];
         const int first_moved = min(first_evicted, len);   // block rows always move into the cache
         const int skip_local = first_moved - seg_a;        // local rows below this keep their place
@@ -1109,7 +973,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 if (lane == 0 && un < p.U) issue_tile(p.k_cache, p.new_k, un, len, B, N, sl, tile, rows_sa, mbar_sa);
             }
         }
-        }   // kSlots
         __syncthreads();   // dst_of is free for the next unit's reduction scratch
     }
     cluster_sync_all();   // no CTA leaves while a peer may still address its shared memory

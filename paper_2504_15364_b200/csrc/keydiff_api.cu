@@ -67,8 +67,6 @@ struct keydiff_ctx {
     int32_t* pos = nullptr;           // [U][N]
     long long next_pos = 0;
     bool pos_stale = true;            // pos must be reset to the identity before the next step uses it
-    int32_t* slot_of = nullptr;       // [U][max_block], fused path: the freed slots of a step, in order
-    int32_t* blk_of = nullptr;        // [U][max_block], fused path: the kept block rows of a step, in order
     void* stage_k = nullptr;          // [U][max_block][128] bf16, keydiff_evict_host only
     void* stage_v = nullptr;
 };
@@ -78,7 +76,7 @@ namespace {
 void free_scratch(keydiff_ctx* c) {
     cudaFree(c->partial); cudaFree(c->norms); cudaFree(c->scores); cudaFree(c->kept_idx);
     cudaFree(c->first_evicted); cudaFree(c->status); cudaFree(c->moved_rows); cudaFree(c->stage_k); cudaFree(c->stage_v);
-    cudaFree(c->anchor_sum[0]); cudaFree(c->anchor_sum[1]); cudaFree(c->anchor_delta); cudaFree(c->pos); cudaFree(c->slot_of); cudaFree(c->blk_of);
+    cudaFree(c->anchor_sum[0]); cudaFree(c->anchor_sum[1]); cudaFree(c->anchor_delta); cudaFree(c->pos);
 }
 
 int check_step_args(const keydiff_ctx* ctx, const void* k_cache, const void* v_cache,
@@ -100,19 +98,17 @@ using FusedKernel = void (*)(kd::FusedParams);
 
 // Kernel instance for `reg_rows` register-resident rows per row group (rounded up to one that is
 // built); one_pass = the variant that takes the anchor from the running sum.
-template <bool kOnePass, bool kSlots>
+template <bool kOnePass>
 FusedKernel fused_instance_of(int reg_rows, int* built) {
     using namespace kd;
-    if (reg_rows <= 0) { *built = 0; return fused_evict_kernel<0, kOnePass, kSlots>; }
-    if (reg_rows <= 2) { *built = 2; return fused_evict_kernel<2, kOnePass, kSlots>; }
-    if (reg_rows <= 4) { *built = 4; return fused_evict_kernel<4, kOnePass, kSlots>; }
-    if (reg_rows <= 5) { *built = 5; return fused_evict_kernel<5, kOnePass, kSlots>; }
-    *built = 6; return fused_evict_kernel<6, kOnePass, kSlots>;
+    if (reg_rows <= 0) { *built = 0; return fused_evict_kernel<0, kOnePass>; }
+    if (reg_rows <= 2) { *built = 2; return fused_evict_kernel<2, kOnePass>; }
+    if (reg_rows <= 4) { *built = 4; return fused_evict_kernel<4, kOnePass>; }
+    if (reg_rows <= 5) { *built = 5; return fused_evict_kernel<5, kOnePass>; }
+    *built = 6; return fused_evict_kernel<6, kOnePass>;
 }
-// slots = the variant with unordered slot reuse
-FusedKernel fused_instance(int reg_rows, int* built, bool one_pass = false, bool slots = false) {
-    if (slots) return one_pass ? fused_instance_of<true, true>(reg_rows, built) : fused_instance_of<false, true>(reg_rows, built);
-    return one_pass ? fused_instance_of<true, false>(reg_rows, built) : fused_instance_of<false, false>(reg_rows, built);
+FusedKernel fused_instance(int reg_rows, int* built, bool one_pass = false) {
+    return one_pass ? fused_instance_of<true>(reg_rows, built) : fused_instance_of<false>(reg_rows, built);
 }
 
 // Co-resident clusters of `C` CTAs of the kernel `kern` with `smem` bytes each.
@@ -157,7 +153,7 @@ bool plan_fused(keydiff_ctx* c, int sm_count) {
         if (sr + kMaxRegRows * kGroups < per_cta) continue;          // slice too long for this cluster size
         const int smem = fused_layout(sr, nkeys, C).total;
         int reg_rows = 0;
-        const FusedKernel kern = fused_instance((std::max(0, per_cta - sr) + kGroups - 1) / kGroups, &reg_rows, false, slot_reuse(c));
+        const FusedKernel kern = fused_instance((std::max(0, per_cta - sr) + kGroups - 1) / kGroups, &reg_rows);
         const int clusters = max_active_clusters(kern, C, smem, sm_count);
         if (clusters < 1) continue;
         const int used = std::min(c->U, clusters);
@@ -171,8 +167,8 @@ bool plan_fused(keydiff_ctx* c, int sm_count) {
     if (!found) return false;
     // the attributes of the chosen instance (the loop may have left another size's values behind)
     int built = 0;
-    return max_active_clusters(fused_instance(c->fused_reg_rows, &built, false, slot_reuse(c)), c->cluster, c->fused_smem_bytes, sm_count) >= 1 &&
-           max_active_clusters(fused_instance(c->fused_reg_rows, &built, true, slot_reuse(c)), c->cluster, c->fused_smem_bytes, sm_count) >= 1;
+    return max_active_clusters(fused_instance(c->fused_reg_rows, &built, false), c->cluster, c->fused_smem_bytes, sm_count) >= 1 &&
+           max_active_clusters(fused_instance(c->fused_reg_rows, &built, true), c->cluster, c->fused_smem_bytes, sm_count) >= 1;
 }
 
 // Slot reuse: cluster size and ring of the streaming kernel for units of up to nmax rows; false if it
@@ -279,8 +275,6 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     p.anchor_delta = c->anchor_delta;
     p.raw_anchor = c->cfg.anchor_mode == KEYDIFF_ANCHOR_RAW_MEAN;
     p.window = c->cfg.recent_window;
-    p.pos = c->pos; p.next_pos = static_cast<int>(c->next_pos);
-    p.slot_of = c->slot_of; p.blk_of = c->blk_of; p.max_block = c->cfg.max_block;
     const int nclusters = std::min(c->U, c->fused_max_clusters);
     // Start-up stagger: somewhat less than one unit's duration spread evenly over the co-resident
     // clusters.  A unit moves 4 slices (K in, K out, V in, V out) per SM at roughly 60 GB/s per SM when
@@ -302,7 +296,7 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     attr[0].val.clusterDim.x = c->cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     int built = 0;
-    KD_CUDA(cudaLaunchKernelEx(&cfg, fused_instance(c->fused_reg_rows, &built, one_pass, slot_reuse(c)), p));
+    KD_CUDA(cudaLaunchKernelEx(&cfg, fused_instance(c->fused_reg_rows, &built, one_pass), p));
     c->anchor_par ^= 1;
     c->anchor_valid = true;
     c->steps_since_full = one_pass ? c->steps_since_full + 1 : 0;
@@ -400,9 +394,9 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
     }
     if (ok) ok = cudaDeviceSynchronize() == cudaSuccess;
     if (ok && cfg->path != KEYDIFF_PATH_STAGED) {
-        const bool use_stream = slot_reuse(c) && !std::getenv("KEYDIFF_SLOT_RESIDENT") && plan_slot_stream(c, prop.multiProcessorCount);
-        c->slot_stream = use_stream;
-        if (use_stream || plan_fused(c, prop.multiProcessorCount)) {
+        // slot reuse is served by the streaming kernel (or, where that cannot hold a unit's keys, by the staged path)
+        c->slot_stream = slot_reuse(c) && plan_slot_stream(c, prop.multiProcessorCount);
+        if (c->slot_stream || (!slot_reuse(c) && plan_fused(c, prop.multiProcessorCount))) {
             c->path = KEYDIFF_PATH_FUSED;
             const size_t sum_bytes = sizeof(double) * U * kd::kHeadDim;
             ok = cudaMalloc(&c->anchor_sum[0], sum_bytes) == cudaSuccess && cudaMalloc(&c->anchor_sum[1], sum_bytes) == cudaSuccess &&
@@ -410,12 +404,6 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
                  cudaMemset(c->anchor_sum[0], 0, sum_bytes) == cudaSuccess && cudaMemset(c->anchor_sum[1], 0, sum_bytes) == cudaSuccess &&
                  cudaMemset(c->anchor_delta, 0, sizeof(float) * U * c->cluster * kd::kHeadDim) == cudaSuccess &&
                  cudaDeviceSynchronize() == cudaSuccess;
-            if (ok && slot_reuse(c)) {
-                const size_t list_bytes = sizeof(int32_t) * U * cfg->max_block;
-                ok = cudaMalloc(&c->slot_of, list_bytes) == cudaSuccess && cudaMalloc(&c->blk_of, list_bytes) == cudaSuccess &&
-                     cudaMemset(c->slot_of, 0, list_bytes) == cudaSuccess && cudaMemset(c->blk_of, 0, list_bytes) == cudaSuccess &&
-                     cudaDeviceSynchronize() == cudaSuccess;
-            }
             if (const char* env = std::getenv("KEYDIFF_INCREMENTAL")) c->incremental = env[0] != '0';   // tuning aid
         } else if (cfg->path == KEYDIFF_PATH_FUSED) {
             free_scratch(c);

@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
     int* blk_of = slot_of + p.max_block;                   // kept block rows, ascending
     SelectSmem& sel = *reinterpret_cast<SelectSmem*>(smem + L.sel);
     float* mu_sh = reinterpret_cast<float*>(smem + L.mu);
-    int* misc = reinterpret_cast<int*>(smem + L.misc);   // 0 ncand, 1 first evicted, 2 need_eq, 3 threshold key, 4 evicted cache rows
+    int* misc = reinterpret_cast<int*>(smem + L.misc);   // 0 ncand, 1 first evicted, 2 need_eq, 3 threshold key, 5/6 prefix carry
     const uint32_t ring_sa = smem_addr(ring), mbar_sa = smem_addr(smem + L.mbar), keys_sa = smem_addr(keys);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = tid >> 3, t = tid & 7, sub = lane >> 3;
@@ -345,7 +345,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
             // the full-table select writes the same bitmap (cleared first: the attempt above may have marked some)
             for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;
             __syncthreads();
-            full_select_plan(keys, n, N, 0, 0, hist, cand_key, cand_idx, nullptr, sel, misc, len, bitmap);
+            full_select_plan(keys, n, N, 0, 0, hist, cand_key, cand_idx, nullptr, sel, misc, bitmap);
         }
         {
             // evicted candidates before each word of the bitmap
@@ -411,32 +411,37 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
             float2 gone[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q) gone[q] = make_float2(0.f, 0.f);
-            const int todo = max(E, kb);
-            for (int r0 = 0; r0 < todo; r0 += C * kGroups) {   // (same trip count in every lane: row_a1 shuffles)
-                const int r = r0 + crank * kGroups + g;
-                const bool ev = r < E;
-                if (__any_sync(0xffffffffu, ev)) {
-                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
-                    if (ev) {
-                        const uint4* row = concat_row(p.k_cache, p.new_k, u, ev_of[r], len, B, N);
-                        a = row[t]; b = row[t + 8];
-                    }
-                    row_a1(a, b, ev, inv_eps, gone, raw);
+            // (a) evicted rows, read once more (from L2); the next row is requested before this one is used
+            const int stride = C * kGroups, r_first = crank * kGroups + g;
+            uint4 na = make_uint4(0, 0, 0, 0), nb = na;
+            if (r_first < E) {
+                const uint4* row = concat_row(p.k_cache, p.new_k, u, ev_of[r_first], len, B, N);
+                na = row[t]; nb = row[t + 8];
+            }
+            for (int r0 = 0; r0 < E; r0 += stride) {   // (same trip count in every lane: row_a1 shuffles)
+                const int r = r0 + r_first;
+                const uint4 a = na, b = nb;
+                if (r + stride < E) {
+                    const uint4* row = concat_row(p.k_cache, p.new_k, u, ev_of[r + stride], len, B, N);
+                    na = row[t]; nb = row[t + 8];
                 }
-                if (r < kb) {
-                    // freed slot r is evicted cache row r for r < evicted_cache: the lanes that read its old words
-                    // above are the ones that overwrite them here
-                    const int slot = slot_of[r], j = blk_of[r];
-                    const uint4* sk = p.new_k + (static_cast<size_t>(u) * B + j) * kRowVec;
-                    const uint4* sv = p.new_v + (static_cast<size_t>(u) * B + j) * kRowVec;
-                    uint4* dk = p.k_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
-                    uint4* dv = p.v_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
-                    dk[t] = sk[t]; dk[t + 8] = sk[t + 8];
-                    dv[t] = sv[t]; dv[t + 8] = sv[t + 8];
-                    if (t == 0) {
-                        p.kept_idx[static_cast<size_t>(u) * N + slot] = len + j;
-                        p.pos[static_cast<size_t>(u) * N + slot] = p.next_pos + j;
-                    }
+                row_a1(a, b, r < E, inv_eps, gone, raw);   // (a row past the end is all zeros and is not added)
+            }
+            // (b) kept block row r into freed slot r.  For r < evicted_cache that slot is evicted row r, whose
+            // old words the same lanes read in (a): a lane's own load and store to one address stay in order.
+#pragma unroll 2
+            for (int r = r_first; r < kb; r += stride) {
+                const int slot = slot_of[r], j = blk_of[r];
+                const uint4* sk = p.new_k + (static_cast<size_t>(u) * B + j) * kRowVec;
+                const uint4* sv = p.new_v + (static_cast<size_t>(u) * B + j) * kRowVec;
+                uint4* dk = p.k_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
+                uint4* dv = p.v_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
+                const uint4 k0 = sk[t], k1 = sk[t + 8], v0 = sv[t], v1 = sv[t + 8];
+                dk[t] = k0; dk[t + 8] = k1;
+                dv[t] = v0; dv[t + 8] = v1;
+                if (t == 0) {
+                    p.kept_idx[static_cast<size_t>(u) * N + slot] = len + j;
+                    p.pos[static_cast<size_t>(u) * N + slot] = p.next_pos + j;
                 }
             }
             float* red2 = reinterpret_cast<float*>(keys);   // the key table is dead until the next unit
