@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (bytes per step of the named workload); None = not captured.
-NCU_TRAFFIC_BYTES = {"llama31_8b_n8192": 2.1111e9}
+NCU_TRAFFIC_BYTES = {("llama31_8b_n8192", "ordered"): 2.1111e9, ("llama31_8b_n8192", "slot_reuse"): 5.918e8}
 
 
 def measured_peak():
@@ -49,12 +49,16 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
-def algorithmic_bytes(wl, moved_rows_per_step_per_unit: float) -> float:
+def algorithmic_bytes(wl, moved_rows_per_step_per_unit: float, slot_reuse: bool = False) -> float:
     """Bytes one evicting step must move: every key read once, moved K rows written, moved V rows
-    read and written, fp32 scores written once and read once."""
+    read and written, fp32 scores written once and read once.  With slot reuse only the kept block
+    rows move (K and V, read and written), and the scores and the slot list are written once."""
     row = wl.head_dim * 2
     n = wl.budget + wl.block
-    per_unit = n * row + 3.0 * moved_rows_per_step_per_unit * row + 2 * n * 4
+    if slot_reuse:
+        per_unit = n * row + 4.0 * moved_rows_per_step_per_unit * row + n * 4 + wl.budget * 4
+    else:
+        per_unit = n * row + 3.0 * moved_rows_per_step_per_unit * row + 2 * n * 4
     return wl.units * per_unit
 
 
@@ -118,7 +122,9 @@ def run_ours(args):
     stream = synth.KVStream(wl, dev, rank=rank)
     k_cache = torch.zeros(U, N, d, dtype=torch.bfloat16, device=dev)
     v_cache = torch.zeros_like(k_cache)
-    kd = KeyDiff(wl.n_layers, wl.batch, wl.n_kv_heads, d, N, B, path=path, device=local)
+    slots = args.compaction == "slot_reuse"
+    kd = KeyDiff(wl.n_layers, wl.batch, wl.n_kv_heads, d, N, B, path=path, device=local,
+                 compaction=binding.KEYDIFF_COMPACT_SLOT_REUSE if slots else binding.KEYDIFF_COMPACT_ORDERED)
     info = kd.launch_info()
     # fill through the library's append path (C_0 = empty)
     for _ in range(wl.fill_steps):
@@ -181,12 +187,13 @@ def run_ours(args):
     if rank != 0:
         return
     peak, peak_src = measured_peak()
-    a_step = algorithmic_bytes(wl, moved)
+    a_step = algorithmic_bytes(wl, moved, slots)
     kern_ms = float(step_ms.mean())
     achieved = a_step / (kern_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get(args.workload), "peak_source": peak_src,
-                "kernel": "fused_evict_kernel" if info["path"] == binding.KEYDIFF_PATH_FUSED else "staged chain (4 kernels)",
+                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, args.compaction)), "peak_source": peak_src,
+                "kernel": ("slot_evict_kernel" if slots else "fused_evict_kernel") if info["path"] == binding.KEYDIFF_PATH_FUSED
+                          else "staged chain (4 kernels)",
                 "algorithmic_bytes_per_launch": a_step, "moved_rows_per_unit": moved,
                 "kernel_ms": kern_ms, "kernel_ms_median": float(np.median(step_ms)),
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
@@ -197,11 +204,17 @@ def run_ours(args):
         from oracle import compare, oracle
         nk, nv = stream.next_block()
         pre_k, pre_v = bits(k_cache), bits(v_cache)
+        if slots:
+            pos_t, next_pos = kd.positions()
+            pre_pos = pos_t.cpu().numpy().astype(np.int64)
         cores = len(os.sched_getaffinity(0))
         times, used = [], 1
         for rep in range(3):
             t0 = time.perf_counter()
-            out = oracle.evict_units_bf16(pre_k, pre_v, N, bits(nk), bits(nv), N, n_threads=cores)
+            if slots:
+                out = oracle.evict_units_bf16_slots(pre_k, pre_v, pre_pos, N, next_pos, bits(nk), bits(nv), N, n_threads=cores)
+            else:
+                out = oracle.evict_units_bf16(pre_k, pre_v, N, bits(nk), bits(nv), N, n_threads=cores)
             times.append(time.perf_counter() - t0)
             used = out["threads"]
             if sum(times) > 12:
@@ -212,8 +225,13 @@ def run_ours(args):
         torch.cuda.synchronize()
         sc = kd.scratch()
         units = np.unique(np.linspace(0, U - 1, 16).astype(int))
-        rep = compare.check_step(pre_k, pre_v, N, bits(nk), bits(nv), N, bits(k_cache), bits(v_cache),
-                                 sc["scores"].cpu().numpy(), sc["kept_idx"].cpu().numpy(), units=units, n_threads=cores)
+        if slots:
+            rep = compare.check_step_slots(pre_k, pre_v, pre_pos, next_pos, N, bits(nk), bits(nv), N, bits(k_cache), bits(v_cache),
+                                           sc["scores"].cpu().numpy(), sc["kept_idx"].cpu().numpy(),
+                                           kd.positions()[0].cpu().numpy(), units=units, n_threads=cores)
+        else:
+            rep = compare.check_step(pre_k, pre_v, N, bits(nk), bits(nv), N, bits(k_cache), bits(v_cache),
+                                     sc["scores"].cpu().numpy(), sc["kept_idx"].cpu().numpy(), units=units, n_threads=cores)
         cpu["parity_units_checked"] = rep["units"]
         cpu["max_score_err_over_tol"] = rep["max_score_err_over_tol"]
 
@@ -224,7 +242,7 @@ def run_ours(args):
                        "head_dim": d, "budget_N": N, "block_B": B, "units": U, "key_model": wl.key_model, "storage_dtype": "bf16",
                        "cache_bytes": 2 * U * N * d * 2, "l2_policy": "inputs larger than L2 (cache >> 126 MB)",
                        "path": "fused" if info["path"] == binding.KEYDIFF_PATH_FUSED else "staged",
-                       "cluster_size": info["cluster_size"], "replicas": world},
+                       "cluster_size": info["cluster_size"], "replicas": world, "compaction": args.compaction},
             "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": K * info["launches_per_step"],
             "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line))
@@ -276,6 +294,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama31_8b_n8192", choices=list(synth.WORKLOADS))
     ap.add_argument("--path", default="auto", choices=["auto", "staged", "fused"])
+    ap.add_argument("--compaction", default="ordered", choices=["ordered", "slot_reuse"],
+                    help="layout of the kept rows: token order (the headline configuration) or unordered slot reuse")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -223,7 +223,8 @@ KEYDIFF_API int keydiff_get_positions(const keydiff_ctx* ctx, const int32_t** po
 KEYDIFF_API int keydiff_get_moved_rows(const keydiff_ctx* ctx, const unsigned long long** counter);
 
 /* Launch facts of the chosen path, for benchmarks: path actually used (KEYDIFF_PATH_*),
- * kernels launched per evicting step, cluster size (1 for the staged path). */
+ * kernels launched per evicting step, cluster size (1 for the staged path).  With slot reuse on the fused
+ * path a step that has to rebuild the running anchor sum (keydiff_set_incremental) launches two more. */
 KEYDIFF_API int keydiff_get_launch_info(const keydiff_ctx* ctx, int32_t* path, int32_t* launches_per_step,
                             int32_t* cluster_size);
 
