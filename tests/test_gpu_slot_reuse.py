@@ -162,3 +162,65 @@ def test_positions_need_the_slot_layout_and_bad_values_are_rejected():
     with pytest.raises(KeyDiffError) as e:
         KeyDiff(1, 1, 2, 128, 64, 8, compaction=3)
     assert e.value.code == binding.KEYDIFF_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_rebuilding_the_anchor_every_step_and_reset(path):
+    # set_incremental(False): the running sum is rebuilt from the cache rows before every step; reset starts a
+    # new sequence (positions from 0 again); both give oracle-exact steps
+    U, N, B = 3, 384, 32
+    k_cache, v_cache, stream = state(U, N, B, N, seed=21, model="outlier")
+    kd = KeyDiff(1, 1, U, 128, N, B, path=path, compaction=SLOTS)
+    kd.set_incremental(False)
+    kd.set_len(N)
+    for step in range(4):
+        checked_step(kd, k_cache, v_cache, *stream.next_block(B), after_set_len=step == 0)
+    kd.set_incremental(True)
+    for step in range(3):
+        checked_step(kd, k_cache, v_cache, *stream.next_block(B))
+    kd.reset()
+    assert kd.len == 0 and kd.positions()[1] == 0
+    for step in range(N // B):
+        kd.evict(k_cache, v_cache, *stream.next_block(B))
+    assert kd.len == N
+    for step in range(3):
+        checked_step(kd, k_cache, v_cache, *stream.next_block(B))
+    kd.close()
+
+
+def test_block_from_host_memory():
+    # keydiff_evict_host with slot reuse: the slot list read back is the one in scratch
+    U, N, B = 4, 512, 64
+    k_cache, v_cache, stream = state(U, N, B, N, seed=33)
+    kd = KeyDiff(1, 1, U, 128, N, B, compaction=SLOTS)
+    kd.set_len(N)
+    kept_h = torch.empty(U, N, dtype=torch.int32).pin_memory()
+    status_h = torch.ones(1, dtype=torch.int32).pin_memory()
+    for step in range(3):
+        nk, nv = stream.next_block(B)
+        pre_k, pre_v = bits(k_cache), bits(v_cache)
+        pre_pos = np.tile(np.arange(N), (U, 1)) if step == 0 else kd.positions()[0].cpu().numpy().astype(np.int64)
+        next_pos = kd.positions()[1]
+        kd.evict_host(k_cache, v_cache, nk.cpu().pin_memory(), nv.cpu().pin_memory(), kept_h, status_h)
+        torch.cuda.synchronize()
+        assert int(status_h.item()) == 0
+        sc = kd.scratch()
+        assert torch.equal(kept_h, sc["kept_idx"].cpu())
+        compare.check_step_slots(pre_k, pre_v, pre_pos, next_pos, N, bits(nk), bits(nv), N, bits(k_cache), bits(v_cache),
+                                 sc["scores"].cpu().numpy(), kept_h.numpy(), kd.positions()[0].cpu().numpy(), n_threads=8)
+    kd.close()
+
+
+def test_decode_cadence_one_token_per_step():
+    # B = 1 at the headline unit shape: every step scores 8193 keys and replaces one slot
+    wl = synth.scaled(synth.WORKLOADS["llama31_8b_n8192"], n_layers=1, n_kv_heads=3, block=1)
+    k_cache, v_cache, stream = synth.prefilled_cache(wl, DEV)
+    kd = KeyDiff(1, 1, 3, 128, wl.budget, 1, compaction=SLOTS)
+    kd.set_len(wl.budget)
+    for step in range(6):
+        nk, nv = stream.next_block(1)
+        if step in (0, 1, 5):
+            checked_step(kd, k_cache, v_cache, nk, nv, after_set_len=step == 0)
+        else:
+            kd.evict(k_cache, v_cache, nk, nv)
+    kd.close()
