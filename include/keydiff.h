@@ -152,11 +152,16 @@ KEYDIFF_API int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache,
 /*
  * keydiff_evict_host -- the same step with the BLOCK in host memory (the caches stay on
  * the device): copies new_k/new_v (host, block_B rows per unit, same layout) to ctx-owned
- * device staging on `stream`, runs keydiff_evict, then copies the kept-index list
+ * device staging, runs keydiff_evict on `stream`, then copies the kept-index list
  * (U*N int32, see keydiff_get_scratch) and the status word back into kept_idx_host /
- * status_host (host; either may be NULL to skip).  Pinned host memory makes the copies
- * asynchronous; the call itself does not synchronise.  The staging buffers are allocated
- * on first use (that first call synchronises and may return ALLOC).
+ * status_host on `stream` (host; either may be NULL to skip).  The block travels on a copy stream
+ * of the ctx into one of two staging sets, and `stream` waits for it: the copy of one call
+ * overlaps the kernels of the call before it.  It starts as soon as the call is made, without
+ * waiting for work queued on `stream`, so the host block must hold its data when the call is made;
+ * it may be reused once the work enqueued on `stream` has completed.  Pinned host memory makes the
+ * copies asynchronous; the call itself does not synchronise.  While `stream` is being captured all
+ * copies stay on `stream`.  Staging buffers, copy stream and events are created on first use (that
+ * first call synchronises and may return ALLOC).
  */
 KEYDIFF_API int keydiff_evict_host(keydiff_ctx* ctx, void* k_cache, void* v_cache,
                        const void* new_k_host, const void* new_v_host,

@@ -68,15 +68,28 @@ struct keydiff_ctx {
     int32_t* pos = nullptr;           // [U][N]
     long long next_pos = 0;
     bool pos_stale = true;            // pos must be reset to the identity before the next step uses it
-    void* stage_k = nullptr;          // [U][max_block][128] bf16, keydiff_evict_host only
-    void* stage_v = nullptr;
+    // keydiff_evict_host only: two sets of staging buffers [U][max_block][128] bf16 filled on a copy stream
+    // of the ctx, so that the block of step i+1 crosses the bus while the kernels of step i run
+    void* stage_k[2] = {nullptr, nullptr};
+    void* stage_v[2] = {nullptr, nullptr};
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr};   // the set's block has arrived
+    cudaEvent_t ev_consumed[2] = {nullptr, nullptr}; // the step that read the set has finished
+    bool consumed_recorded[2] = {false, false};
+    int stage_next = 0;
 };
 
 namespace {
 
 void free_scratch(keydiff_ctx* c) {
     cudaFree(c->partial); cudaFree(c->norms); cudaFree(c->scores); cudaFree(c->kept_idx);
-    cudaFree(c->first_evicted); cudaFree(c->status); cudaFree(c->moved_rows); cudaFree(c->stage_k); cudaFree(c->stage_v);
+    cudaFree(c->first_evicted); cudaFree(c->status); cudaFree(c->moved_rows);
+    for (int b = 0; b < 2; ++b) {
+        cudaFree(c->stage_k[b]); cudaFree(c->stage_v[b]);
+        if (c->ev_copied[b]) cudaEventDestroy(c->ev_copied[b]);
+        if (c->ev_consumed[b]) cudaEventDestroy(c->ev_consumed[b]);
+    }
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     cudaFree(c->anchor_sum[0]); cudaFree(c->anchor_sum[1]); cudaFree(c->anchor_delta); cudaFree(c->pos);
 }
 
@@ -483,22 +496,50 @@ int keydiff_evict_host(keydiff_ctx* ctx, void* k_cache, void* v_cache, const voi
                        int32_t* kept_idx_host, int32_t* status_host, void* stream) {
     if (!ctx || !new_k_host || !new_v_host) return KEYDIFF_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (!ctx->stage_k) {
+    if (!ctx->copy_stream) {
         const size_t bytes = static_cast<size_t>(ctx->U) * ctx->cfg.max_block * kd::kRowBytes;
-        if (cudaMalloc(&ctx->stage_k, bytes) != cudaSuccess || cudaMalloc(&ctx->stage_v, bytes) != cudaSuccess) {
+        bool ok = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+        for (int b = 0; b < 2 && ok; ++b)
+            ok = cudaMalloc(&ctx->stage_k[b], bytes) == cudaSuccess && cudaMalloc(&ctx->stage_v[b], bytes) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&ctx->ev_copied[b], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&ctx->ev_consumed[b], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
             g_last_cuda_error = static_cast<int>(cudaGetLastError());
-            cudaFree(ctx->stage_k); ctx->stage_k = nullptr;
+            for (int b = 0; b < 2; ++b) {
+                cudaFree(ctx->stage_k[b]); cudaFree(ctx->stage_v[b]); ctx->stage_k[b] = ctx->stage_v[b] = nullptr;
+                if (ctx->ev_copied[b]) { cudaEventDestroy(ctx->ev_copied[b]); ctx->ev_copied[b] = nullptr; }
+                if (ctx->ev_consumed[b]) { cudaEventDestroy(ctx->ev_consumed[b]); ctx->ev_consumed[b] = nullptr; }
+            }
+            if (ctx->copy_stream) { cudaStreamDestroy(ctx->copy_stream); ctx->copy_stream = nullptr; }
             return KEYDIFF_ERR_ALLOC;
         }
     }
-    const int rc = check_step_args(ctx, k_cache, v_cache, ctx->stage_k, ctx->stage_v, budget_N, block_B, n_kv_heads, head_dim);
+    const int b = ctx->stage_next;
+    const int rc = check_step_args(ctx, k_cache, v_cache, ctx->stage_k[b], ctx->stage_v[b], budget_N, block_B, n_kv_heads, head_dim);
     if (rc != KEYDIFF_OK) return rc;
     const size_t bytes = static_cast<size_t>(ctx->U) * block_B * kd::kRowBytes;
-    KD_CUDA(cudaMemcpyAsync(ctx->stage_k, new_k_host, bytes, cudaMemcpyHostToDevice, st));
-    KD_CUDA(cudaMemcpyAsync(ctx->stage_v, new_v_host, bytes, cudaMemcpyHostToDevice, st));
-    const int erc = keydiff_evict(ctx, k_cache, v_cache, ctx->stage_k, ctx->stage_v, budget_N, block_B, n_kv_heads,
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    KD_CUDA(cudaStreamIsCapturing(st, &capturing));
+    if (capturing == cudaStreamCaptureStatusNone) {
+        // the copy does not wait for what is queued on `st`: only for the step that last read this set
+        if (ctx->consumed_recorded[b]) KD_CUDA(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_consumed[b], 0));
+        KD_CUDA(cudaMemcpyAsync(ctx->stage_k[b], new_k_host, bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+        KD_CUDA(cudaMemcpyAsync(ctx->stage_v[b], new_v_host, bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+        KD_CUDA(cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
+        KD_CUDA(cudaStreamWaitEvent(st, ctx->ev_copied[b], 0));
+    } else {
+        // inside a stream capture everything stays on the captured stream
+        KD_CUDA(cudaMemcpyAsync(ctx->stage_k[b], new_k_host, bytes, cudaMemcpyHostToDevice, st));
+        KD_CUDA(cudaMemcpyAsync(ctx->stage_v[b], new_v_host, bytes, cudaMemcpyHostToDevice, st));
+    }
+    const int erc = keydiff_evict(ctx, k_cache, v_cache, ctx->stage_k[b], ctx->stage_v[b], budget_N, block_B, n_kv_heads,
                                   head_dim, stream);
     if (erc != KEYDIFF_OK) return erc;
+    if (capturing == cudaStreamCaptureStatusNone) {
+        KD_CUDA(cudaEventRecord(ctx->ev_consumed[b], st));
+        ctx->consumed_recorded[b] = true;
+    }
+    ctx->stage_next = b ^ 1;
     if (kept_idx_host)
         KD_CUDA(cudaMemcpyAsync(kept_idx_host, ctx->kept_idx, sizeof(int32_t) * ctx->U * ctx->cfg.budget,
                                 cudaMemcpyDeviceToHost, st));

@@ -323,3 +323,28 @@ def test_host_block_entry_point(path):
     assert torch.equal(k_cache, k2) and torch.equal(v_cache, v2)
     assert torch.equal(kept, kd.scratch()["kept_idx"].cpu()) and int(status.item()) == 0
     kd.close(); kd2.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_host_block_calls_back_to_back(path):
+    # six calls queued without a synchronise in between: the block of one call is copied (on the ctx's copy
+    # stream, into alternating staging sets) while the kernels of the call before it run; the caches must
+    # end up exactly as with device-resident blocks
+    wl = synth.Workload("t", 1, 1, 6, 128, 1024, 96, "outlier", 1024 + 6 * 96, 77)
+    k1, v1, stream = synth.prefilled_cache(wl, DEV)
+    k2, v2 = k1.clone(), v1.clone()
+    blocks = [stream.next_block() for _ in range(6)]
+    host = [(a.cpu().pin_memory(), b.cpu().pin_memory()) for a, b in blocks]
+    kd = KeyDiff(1, 1, 6, 128, 1024, 96, path=path); kd.set_len(1024)
+    kd2 = KeyDiff(1, 1, 6, 128, 1024, 96, path=path); kd2.set_len(1024)
+    kept = [torch.empty(6, 1024, dtype=torch.int32).pin_memory() for _ in range(6)]
+    status = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+    for i in range(6):
+        kd2.evict_host(k2, v2, *host[i], kept[i], status)
+    torch.cuda.synchronize()
+    for i in range(6):
+        kd.evict(k1, v1, *blocks[i])
+        torch.cuda.synchronize()
+        assert torch.equal(kept[i], kd.scratch()["kept_idx"].cpu()), i
+    assert torch.equal(k1, k2) and torch.equal(v1, v2) and int(status.item()) == 0
+    kd.close(); kd2.close()
