@@ -160,7 +160,10 @@ KEYDIFF_API int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache,
  * waiting for work queued on `stream`, so the host block must hold its data when the call is made;
  * it may be reused once the work enqueued on `stream` has completed.  Pinned host memory makes the
  * copies asynchronous; the call itself does not synchronise.  While `stream` is being captured all
- * copies stay on `stream`.  Staging buffers, copy stream and events are created on first use (that
+ * copies stay on `stream`.  When kept_idx_host is pinned (page-locked) memory and the fused path serves an
+ * evicting step, the kernel writes the list into it directly while it runs (through the buffer's device
+ * alias) instead of a copy afterwards; either way the list is complete once the work on `stream` is.
+ * Staging buffers, copy stream and events are created on first use (that
  * first call synchronises and may return ALLOC).
  */
 KEYDIFF_API int keydiff_evict_host(keydiff_ctx* ctx, void* k_cache, void* v_cache,

@@ -96,6 +96,7 @@ struct FusedParams {
     const double* anchor_in; double* anchor_out; float* anchor_delta;
     int raw_anchor;     // 1: the anchor is the mean of the keys themselves (Sec. 3.2), 0: of the normalised keys
     int window;         // w most recent tokens that are never evicted (Sec. 3.2, sliding window)
+    int32_t* kept_mirror;   // optional second destination of the kept-index list (device alias of pinned host memory)
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -852,7 +853,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         }
         for (int lr = tid; lr < seg; lr += kFusedThreads) {
             const int d = dst_of[lr];
-            if (d >= 0) p.kept_idx[static_cast<size_t>(u) * N + d] = seg_a + lr;
+            if (d >= 0) {
+                p.kept_idx[static_cast<size_t>(u) * N + d] = seg_a + lr;
+                if (p.kept_mirror) p.kept_mirror[static_cast<size_t>(u) * N + d] = seg_a + lr;
+            }
         }
         // ------------------------------------------------------------ a4: K rows out, V rows in behind them
         {

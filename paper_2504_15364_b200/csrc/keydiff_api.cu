@@ -77,6 +77,8 @@ struct keydiff_ctx {
     cudaEvent_t ev_consumed[2] = {nullptr, nullptr}; // the step that read the set has finished
     bool consumed_recorded[2] = {false, false};
     int stage_next = 0;
+    int32_t* kept_mirror = nullptr;   // set by keydiff_evict_host around its step: the fused kernels also write the
+                                      // kept-index list there (the caller's pinned buffer), so no copy follows
 };
 
 namespace {
@@ -252,6 +254,7 @@ int launch_slot_stream(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, co
     p.raw_anchor = c->cfg.anchor_mode == KEYDIFF_ANCHOR_RAW_MEAN;
     p.window = c->cfg.recent_window;
     p.pos = c->pos; p.next_pos = static_cast<int>(c->next_pos);
+    p.kept_mirror = c->kept_mirror;
     const int nclusters = std::min(c->U, c->fused_max_clusters);
     // Start-up stagger: clusters launched together stream together and then select together, leaving HBM
     // idle in between.  When every cluster serves at least three units, starting cluster c a little later
@@ -300,6 +303,7 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     p.anchor_delta = c->anchor_delta;
     p.raw_anchor = c->cfg.anchor_mode == KEYDIFF_ANCHOR_RAW_MEAN;
     p.window = c->cfg.recent_window;
+    p.kept_mirror = c->kept_mirror;
     const int nclusters = std::min(c->U, c->fused_max_clusters);
     // Start-up stagger: somewhat less than one unit's duration spread evenly over the co-resident
     // clusters.  A unit moves 4 slices (K in, K out, V in, V out) per SM at roughly 60 GB/s per SM when
@@ -532,15 +536,28 @@ int keydiff_evict_host(keydiff_ctx* ctx, void* k_cache, void* v_cache, const voi
         KD_CUDA(cudaMemcpyAsync(ctx->stage_k[b], new_k_host, bytes, cudaMemcpyHostToDevice, st));
         KD_CUDA(cudaMemcpyAsync(ctx->stage_v[b], new_v_host, bytes, cudaMemcpyHostToDevice, st));
     }
+    // Pinned host memory has a device alias: on the fused path an evicting step writes the kept-index list
+    // there itself, as it writes it to scratch, so the list crosses the bus during the step
+    bool mirrored = false;
+    if (kept_idx_host && ctx->path == KEYDIFF_PATH_FUSED && ctx->len + block_B > ctx->cfg.budget) {
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, kept_idx_host) == cudaSuccess && attr.type == cudaMemoryTypeHost && attr.devicePointer) {
+            ctx->kept_mirror = static_cast<int32_t*>(attr.devicePointer);
+            mirrored = true;
+        } else {
+            cudaGetLastError();
+        }
+    }
     const int erc = keydiff_evict(ctx, k_cache, v_cache, ctx->stage_k[b], ctx->stage_v[b], budget_N, block_B, n_kv_heads,
                                   head_dim, stream);
+    ctx->kept_mirror = nullptr;
     if (erc != KEYDIFF_OK) return erc;
     if (capturing == cudaStreamCaptureStatusNone) {
         KD_CUDA(cudaEventRecord(ctx->ev_consumed[b], st));
         ctx->consumed_recorded[b] = true;
     }
     ctx->stage_next = b ^ 1;
-    if (kept_idx_host)
+    if (kept_idx_host && !mirrored)
         KD_CUDA(cudaMemcpyAsync(kept_idx_host, ctx->kept_idx, sizeof(int32_t) * ctx->U * ctx->cfg.budget,
                                 cudaMemcpyDeviceToHost, st));
     if (status_host)

@@ -66,6 +66,7 @@ struct SlotParams {
     int raw_anchor, window;
     int32_t* pos;       // [U][N] token position of every slot
     int next_pos;       // position of the block's first token
+    int32_t* kept_mirror;   // optional second destination of the slot list (device alias of pinned host memory)
 };
 
 // One thread: bulk-load unit rows [g0, g0 + nrows) of unit u (cache rows below len, block rows after) to dst.
@@ -396,7 +397,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
         for (int e = len + tid; e < N; e += kFusedThreads) slot_of[evicted_cache + (e - len)] = e;   // slots that were still empty
         // kept cache rows of this slice keep their slot: the kept-index list says so
         for (int i = seg_a + tid; i < min(seg_b, len); i += kFusedThreads)
-            if (!((bitmap[i >> 5] >> (i & 31)) & 1u)) p.kept_idx[static_cast<size_t>(u) * N + i] = i;
+            if (!((bitmap[i >> 5] >> (i & 31)) & 1u)) {
+                p.kept_idx[static_cast<size_t>(u) * N + i] = i;
+                if (p.kept_mirror) p.kept_mirror[static_cast<size_t>(u) * N + i] = i;
+            }
         if (crank == 0 && tid == 0) {
             p.first_evicted[u] = misc[1];
             atomicAdd(p.moved_rows, static_cast<unsigned long long>(kb));
@@ -441,6 +445,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
                 dv[t] = v0; dv[t + 8] = v1;
                 if (t == 0) {
                     p.kept_idx[static_cast<size_t>(u) * N + slot] = len + j;
+                    if (p.kept_mirror) p.kept_mirror[static_cast<size_t>(u) * N + slot] = len + j;
                     p.pos[static_cast<size_t>(u) * N + slot] = p.next_pos + j;
                 }
             }
