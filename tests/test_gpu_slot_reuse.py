@@ -224,3 +224,53 @@ def test_decode_cadence_one_token_per_step():
         else:
             kd.evict(k_cache, v_cache, nk, nv)
     kd.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_all_keys_identical_nothing_is_written(path):
+    # every score ties: the lower candidate numbers (the cache slots) stay, every block row goes, no slot changes
+    U, N, B = 2, 200, 40
+    row = torch.randn(1, 1, 128, generator=torch.Generator().manual_seed(1)).to(torch.bfloat16)
+    k_cache = row.expand(U, N, 128).contiguous().to(DEV); new_k = row.expand(U, B, 128).contiguous().to(DEV)
+    tag = torch.arange(N + B, dtype=torch.float32).view(1, -1, 1).expand(U, N + B, 128).to(torch.bfloat16)
+    v_cache = tag[:, :N].contiguous().to(DEV); new_v = tag[:, N:].contiguous().to(DEV)
+    before_k, before_v = k_cache.clone(), v_cache.clone()
+    kd = KeyDiff(1, 1, U, 128, N, B, path=path, compaction=SLOTS)
+    kd.set_len(N)
+    checked_step(kd, k_cache, v_cache, new_k, new_v, after_set_len=True)
+    assert (kd.scratch()["kept_idx"].cpu().numpy() == np.arange(N)).all()
+    assert torch.equal(k_cache, before_k) and torch.equal(v_cache, before_v)
+    assert (kd.positions()[0].cpu().numpy() == np.arange(N)).all() and kd.positions()[1] == N + B
+    kd.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_zero_anchor_and_zero_keys(path):
+    # antipodal pairs cancel the anchor exactly (all scores 0 -> candidate-number tie-break); plus zero keys
+    U, N, B = 1, 64, 16
+    g = torch.Generator().manual_seed(2)
+    half = torch.randn(U, (N + B) // 2, 128, generator=g).to(torch.bfloat16)
+    allk = torch.cat([half, -half], dim=1)
+    allk[:, 5] = 0; allk[:, 5 + (N + B) // 2] = 0
+    v = torch.randn(U, N + B, 128, generator=g).to(torch.bfloat16)
+    k_cache, new_k = allk[:, :N].contiguous().to(DEV), allk[:, N:].contiguous().to(DEV)
+    v_cache, new_v = v[:, :N].contiguous().to(DEV), v[:, N:].contiguous().to(DEV)
+    kd = KeyDiff(1, 1, U, 128, N, B, path=path, compaction=SLOTS)
+    kd.set_len(N)
+    rep = checked_step(kd, k_cache, v_cache, new_k, new_v, after_set_len=True)
+    assert rep["min_anchor_norm"] < 1e-3
+    sc = kd.scratch()["scores"][0, :N + B].cpu().numpy()
+    assert sc[5] == 0.0 and not np.signbit(sc[5])
+    kd.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("model", ["clusters", "drift"])
+def test_key_models(path, model):
+    wl = synth.Workload("t", 1, 2, 3, 128, 1024, 128, model, 1024 + 8 * 128, 91)
+    k_cache, v_cache, stream = synth.prefilled_cache(wl, DEV)
+    kd = KeyDiff(wl.n_layers, wl.batch, wl.n_kv_heads, 128, wl.budget, wl.block, path=path, compaction=SLOTS)
+    kd.set_len(wl.budget)
+    for step in range(8):
+        checked_step(kd, k_cache, v_cache, *stream.next_block(), after_set_len=step == 0)
+    kd.close()
