@@ -59,7 +59,8 @@ struct SlotParams {
     int nwords;         // bitmap words provided for (>= ceil(n / 32))
     int nmax;           // row stride of the score scratch
     int max_block;
-    unsigned stagger_ns;
+    unsigned stagger_ns;   // cluster c starts c * stagger_ns late
+    unsigned late_ns;      // clusters that serve one unit fewer than the others start this much later still
     float* scores; int32_t* kept_idx; int32_t* first_evicted;
     unsigned long long* moved_rows; int32_t* status;
     const double* anchor_in; double* anchor_out; float* anchor_delta;   // running anchor, as in FusedParams
@@ -128,6 +129,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
         const unsigned long long t0 = global_timer_ns();
         const unsigned long long wait_ns = static_cast<unsigned long long>(p.stagger_ns) * static_cast<unsigned>(cluster_id);
         for (int spin = 0; spin < (1 << 16) && global_timer_ns() - t0 < wait_ns; ++spin) __nanosleep(100);
+    }
+    // When the units do not divide evenly, the clusters with one unit fewer have a unit's time to spare: they
+    // start late, so that their stream runs while the others are between streams (selection, placement)
+    // instead of competing with the others' first stream.  Bounded like the wait above.
+    if (p.late_ns != 0 && my_units > 0 && my_units < (p.U + nclusters - 1) / nclusters) {
+        const unsigned long long t0 = global_timer_ns();
+        for (int spin = 0; spin < (1 << 16) && global_timer_ns() - t0 < p.late_ns; ++spin) __nanosleep(200);
     }
 
     // issue side of the warp's stream: the next tile to request is tile i_j of the cluster's i_it-th unit
@@ -208,6 +216,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
                 for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
                 m = sqrtf(v);
             }
+            float* sc = p.scores + static_cast<size_t>(u) * p.nmax + seg_a;
 #pragma unroll 1
             for (int j = 0; j < cnt_w; ++j) {
                 const int phys = warp + kFusedWarps * c_d;
@@ -225,7 +234,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
                 }
                 const uint32_t key = score4(v, t, m, p.eps);
                 const int lr = lo + (t >> 1) * 4 + sub;
-                if (!(t & 1) && lr < seg) keys[seg_a + lr] = key;
+                if (!(t & 1) && lr < seg) {
+                    keys[seg_a + lr] = key;
+                    sc[lr] = key_score(key);   // fp32 score to global scratch: the tile's 16 scores are one 64-byte line
+                }
                 __syncwarp();   // the tile's only readers are this warp's lanes: the copy engine may refill it
                 if (lane == 0 && i_it < my_units) issue_next(c_d);
                 if (++c_d == D) c_d = 0;
@@ -244,8 +256,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
             cluster_arrive();
         }
         {
-            float* sc = p.scores + static_cast<size_t>(u) * p.nmax + seg_a;   // fp32 scores to global scratch, coalesced
-            for (int lr = tid; lr < seg; lr += kFusedThreads) sc[lr] = key_score(keys[seg_a + lr]);
             for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;
             for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;
             if (tid == 0) { misc[0] = 0; misc[1] = n; }
