@@ -769,7 +769,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             // bin of a key: linear in the key over [kmin, kcut] (bins 0..2046), 2047 above; monotone
             auto bin_of = [kmin, kcut, shift](uint32_t k) { return k <= kcut ? min((k - kmin) >> shift, 2046u) : 2047u; };
 #pragma unroll
-            for (int j = 0; j < kFastKeys; ++j) if (j < cnt) atomicAdd(&hist[bin_of(kk[j])], 1);
+            for (int j = 0; j < kFastKeys; ++j) {
+                // (the top bin holds every key above the bound: the crossing is never there, so it is not counted)
+                const uint32_t b = bin_of(kk[j]);
+                if (j < cnt && b != 2047u) atomicAdd(&hist[b], 1);
+            }
             __syncthreads();
             const int packed = find_crossing(hist, E, lane, warp, sel.warp_eq);
             const uint32_t bstar = static_cast<uint32_t>(packed >> 16);
@@ -781,19 +785,22 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 m_below |= (j < cnt && b < bstar) ? 1u << j : 0u;
                 m_in |= (j < cnt && b == bstar) ? 1u << j : 0u;
             }
-            if (packed >= 0 && (m_below | m_in)) {
+            {
                 int first = n;
-                for (unsigned m = m_below; m; m &= m - 1) {
-                    const int i = tid + (__ffs(m) - 1) * kFusedThreads;
-                    atomicOr(&bitmap[i >> 5], 1u << (i & 31));
-                    first = min(first, i);
+                if (packed >= 0 && (m_below | m_in)) {
+                    for (unsigned m = m_below; m; m &= m - 1) {
+                        const int i = tid + (__ffs(m) - 1) * kFusedThreads;
+                        atomicOr(&bitmap[i >> 5], 1u << (i & 31));
+                        first = min(first, i);
+                    }
+                    for (unsigned m = m_in; m; m &= m - 1) {
+                        const int i = tid + (__ffs(m) - 1) * kFusedThreads;
+                        const int slot = atomicAdd(&misc[0], 1);
+                        if (slot < kFastCandCap) { fcand_key[slot] = keys[i]; fcand_idx[slot] = i; }
+                    }
                 }
-                for (unsigned m = m_in; m; m &= m - 1) {
-                    const int i = tid + (__ffs(m) - 1) * kFusedThreads;
-                    const int slot = atomicAdd(&misc[0], 1);
-                    if (slot < kFastCandCap) { fcand_key[slot] = keys[i]; fcand_idx[slot] = i; }
-                }
-                if (first < n) atomicMin(&misc[1], first);
+                first = __reduce_min_sync(0xffffffffu, first);   // one shared-memory atomic per warp, not per thread
+                if (lane == 0 && first < n) atomicMin(&misc[1], first);
             }
             __syncthreads();
             const int ncand = misc[0];

@@ -306,7 +306,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
             }
             auto bin_of = [kmin, kcut, shift](uint32_t k) { return k <= kcut ? min((k - kmin) >> shift, 2046u) : 2047u; };
 #pragma unroll
-            for (int j = 0; j < kFastKeys; ++j) if (j < cnt) atomicAdd(&hist[bin_of(kk[j])], 1);
+            for (int j = 0; j < kFastKeys; ++j) {
+                // (the top bin holds every key above the bound: the crossing is never there, so it is not counted)
+                const uint32_t b = bin_of(kk[j]);
+                if (j < cnt && b != 2047u) atomicAdd(&hist[b], 1);
+            }
             __syncthreads();
             const int packed = find_crossing(hist, E, lane, warp, sel.warp_eq);
             const uint32_t bstar = static_cast<uint32_t>(packed >> 16);
@@ -318,19 +322,22 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
                 m_below |= (j < cnt && b < bstar) ? 1u << j : 0u;
                 m_in |= (j < cnt && b == bstar) ? 1u << j : 0u;
             }
-            if (packed >= 0 && (m_below | m_in)) {
+            {
                 int first = n;
-                for (unsigned mm = m_below; mm; mm &= mm - 1) {
-                    const int i = tid + (__ffs(mm) - 1) * kFusedThreads;
-                    atomicOr(&bitmap[i >> 5], 1u << (i & 31));
-                    first = min(first, i);
+                if (packed >= 0 && (m_below | m_in)) {
+                    for (unsigned mm = m_below; mm; mm &= mm - 1) {
+                        const int i = tid + (__ffs(mm) - 1) * kFusedThreads;
+                        atomicOr(&bitmap[i >> 5], 1u << (i & 31));
+                        first = min(first, i);
+                    }
+                    for (unsigned mm = m_in; mm; mm &= mm - 1) {
+                        const int i = tid + (__ffs(mm) - 1) * kFusedThreads;
+                        const int slot = atomicAdd(&misc[0], 1);
+                        if (slot < kFastCandCap) { cand_key[slot] = keys[i]; cand_idx[slot] = i; }
+                    }
                 }
-                for (unsigned mm = m_in; mm; mm &= mm - 1) {
-                    const int i = tid + (__ffs(mm) - 1) * kFusedThreads;
-                    const int slot = atomicAdd(&misc[0], 1);
-                    if (slot < kFastCandCap) { cand_key[slot] = keys[i]; cand_idx[slot] = i; }
-                }
-                if (first < n) atomicMin(&misc[1], first);
+                first = __reduce_min_sync(0xffffffffu, first);   // one shared-memory atomic per warp, not per thread
+                if (lane == 0 && first < n) atomicMin(&misc[1], first);
             }
             __syncthreads();
             const int ncand = misc[0];
