@@ -75,7 +75,10 @@ enum {
 enum {
     KEYDIFF_COMPACT_ORDERED = 0,    /* kept rows in original token order, compacted to the front (default) */
     KEYDIFF_COMPACT_SLOT_REUSE = 1  /* kept cache rows stay in their slots; the kept block rows take the
-                                       freed slots: at most block_B rows per tensor are written */
+                                       freed slots: at most block_B rows per tensor are written.  The fused
+                                       path serves it with a streaming kernel for max_block <= 1024; larger
+                                       blocks go to the staged kernels (KEYDIFF_PATH_FUSED then fails with
+                                       KEYDIFF_ERR_UNSUPPORTED) */
 };
 
 /* Which kernels serve keydiff_evict. */

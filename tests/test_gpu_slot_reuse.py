@@ -274,3 +274,18 @@ def test_key_models(path, model):
     for step in range(8):
         checked_step(kd, k_cache, v_cache, *stream.next_block(), after_set_len=step == 0)
     kd.close()
+
+
+def test_blocks_beyond_the_streaming_kernel_go_to_the_staged_path():
+    # the streaming kernel keeps three max_block-sized lists in shared memory and is built for max_block <= 1024
+    U, N, B = 2, 2048, 1500
+    with pytest.raises(KeyDiffError) as e:
+        KeyDiff(1, 1, U, 128, N, B, path=binding.KEYDIFF_PATH_FUSED, compaction=SLOTS)
+    assert e.value.code == binding.KEYDIFF_ERR_UNSUPPORTED
+    kd = KeyDiff(1, 1, U, 128, N, B, compaction=SLOTS)
+    assert kd.launch_info()["path"] == binding.KEYDIFF_PATH_STAGED
+    k_cache, v_cache, stream = state(U, N, B, N, seed=3)
+    kd.set_len(N)
+    for step in range(2):
+        checked_step(kd, k_cache, v_cache, *stream.next_block(B), after_set_len=step == 0)
+    kd.close()
