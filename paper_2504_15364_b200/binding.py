@@ -100,6 +100,9 @@ class KeyDiff:
 
     ``evict`` mirrors ``keydiff_evict``; tensors are bf16 CUDA tensors laid out
     [n_layers, batch, n_kv_heads, rows, head_dim] (or the same flattened to [U, rows, head_dim]).
+    ``anchor_mode`` / ``recent_window`` choose the method's variants (raw-mean anchor, sliding window);
+    ``compaction=KEYDIFF_COMPACT_SLOT_REUSE`` leaves kept cache rows in their slots and writes the kept
+    block rows into the freed ones (``positions()`` then tells which token each slot holds).
     """
 
     def __init__(self, n_layers: int, batch: int, n_kv_heads: int, head_dim: int, budget: int, max_block: int,
