@@ -289,3 +289,15 @@ def test_blocks_beyond_the_streaming_kernel_go_to_the_staged_path():
     for step in range(2):
         checked_step(kd, k_cache, v_cache, *stream.next_block(B), after_set_len=step == 0)
     kd.close()
+
+
+@pytest.mark.parametrize("U,N,B,w", [(3, 9000, 300, 0), (3, 9000, 300, 900), (2, 17000, 400, 0)])
+def test_units_beyond_the_register_select(U, N, B, w):
+    # more than 17 keys per thread: the streaming kernel takes the full-table select, which fills the same
+    # bitmap; beyond 16384 candidates the bitmap's prefix runs over more than one 512-word chunk
+    k_cache, v_cache, stream = state(U, N, B, N, seed=70 + w, model="outlier")
+    kd = KeyDiff(1, 1, U, 128, N, B, path=binding.KEYDIFF_PATH_FUSED, compaction=SLOTS, recent_window=w)
+    kd.set_len(N)
+    for step in range(2):
+        checked_step(kd, k_cache, v_cache, *stream.next_block(B), 0, w, after_set_len=step == 0)
+    kd.close()
