@@ -37,7 +37,8 @@ def test_null_and_bad_config_rejected_before_any_device_work(lib):
     assert lib.keydiff_create(None, ctypes.byref(out)) == binding.KEYDIFF_ERR_INVALID_ARG
     cfg = binding.keydiff_config(1, 1, 8, 128, 512, 128, binding.KEYDIFF_BF16, 0, 0.0, 0)
     assert lib.keydiff_create(ctypes.byref(cfg), None) == binding.KEYDIFF_ERR_INVALID_ARG
-    for field, bad in [("n_layers", 0), ("budget", 0), ("max_block", -1), ("device", -1), ("path", 7)]:
+    for field, bad in [("n_layers", 0), ("budget", 0), ("max_block", -1), ("device", -1), ("path", 7),
+                       ("anchor_mode", 2), ("recent_window", -1), ("recent_window", 513), ("compaction", 2)]:
         c = binding.keydiff_config(1, 1, 8, 128, 512, 128, binding.KEYDIFF_BF16, 0, 0.0, 0)
         setattr(c, field, bad)
         assert lib.keydiff_create(ctypes.byref(c), ctypes.byref(out)) == binding.KEYDIFF_ERR_INVALID_ARG, field
@@ -47,6 +48,7 @@ def test_null_and_bad_config_rejected_before_any_device_work(lib):
     assert lib.keydiff_create(ctypes.byref(c), ctypes.byref(out)) == binding.KEYDIFF_ERR_UNSUPPORTED
     assert lib.keydiff_destroy(None) == binding.KEYDIFF_OK
     assert lib.keydiff_get_len(None, None) == binding.KEYDIFF_ERR_INVALID_ARG
+    assert lib.keydiff_get_positions(None, None, None) == binding.KEYDIFF_ERR_INVALID_ARG
     assert lib.keydiff_evict(None, None, None, None, None, 1, 1, 1, 128, None) == binding.KEYDIFF_ERR_INVALID_ARG
 
 
