@@ -5,7 +5,7 @@ A step is one ``keydiff_evict`` call over all units of the workload for one appe
 steady state (cache at its budget, B rows evicted per unit).  Default workload: the
 Llama-3.1-8B-shaped config (32 layers x 8 KV heads, N=8192, B=128, 32K-token prompt).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--path auto|staged|fused]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--path auto|staged|fused] [--headline-only]
   python bench.py --impl reference ...        # the CPU oracle on the host cores, same metric
 
 Prints ONE JSON line (rank 0).  Under torchrun every rank runs its own replica of the workload
@@ -46,7 +46,7 @@ def measured_peak():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     except Exception:
-        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, an earlier measurement of the same GPU model)"
 
 
 def algorithmic_bytes(wl, moved_rows_per_step_per_unit: float, slot_reuse: bool = False) -> float:
@@ -106,8 +106,139 @@ def bits(t):
     return t.detach().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
+class Run:
+    """One workload on one layout, resident on the device: cache filled through the library's append path."""
+
+    def __init__(self, wl, compaction, path, dev, rank):
+        from paper_2504_15364_b200 import KeyDiff, binding
+        self.wl, self.dev, self.slots = wl, dev, compaction == "slot_reuse"
+        U, N, B, d = wl.units, wl.budget, wl.block, wl.head_dim
+        self.stream = synth.KVStream(wl, dev, rank=rank)
+        self.k_cache = torch.zeros(U, N, d, dtype=torch.bfloat16, device=dev)
+        self.v_cache = torch.zeros_like(self.k_cache)
+        self.kd = KeyDiff(wl.n_layers, wl.batch, wl.n_kv_heads, d, N, B, path=path, device=dev.index,
+                          compaction=binding.KEYDIFF_COMPACT_SLOT_REUSE if self.slots else binding.KEYDIFF_COMPACT_ORDERED)
+        self.info = self.kd.launch_info()
+        self.fused = self.info["path"] == binding.KEYDIFF_PATH_FUSED
+        for _ in range(wl.fill_steps):
+            self.kd.evict(self.k_cache, self.v_cache, *self.stream.next_block())
+        assert self.kd.len == N
+
+    def step(self, block):
+        self.kd.evict(self.k_cache, self.v_cache, *block)
+
+    def timed(self, K, W, sampler=None):
+        """W untimed steps, then K steps timed with CUDA events on the launching stream (one event pair per
+        step); returns total ms, per-step ms, moved rows per unit per step."""
+        blocks = [self.stream.next_block() for _ in range(W + K)]
+        for i in range(W):
+            self.step(blocks[i])
+        torch.cuda.synchronize()
+        moved0 = self.kd.moved_rows()
+        st = torch.cuda.current_stream(self.dev)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+        kdist.barrier()
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.start()
+        ev[0].record(st)
+        for i in range(K):
+            self.step(blocks[W + i])
+            ev[i + 1].record(st)
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.stop_flag = True
+        kdist.barrier()
+        if sampler:
+            sampler.join()
+        step_ms = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(K)])
+        moved = (self.kd.moved_rows() - moved0) / K / self.wl.units
+        status = int(self.kd.scratch()["status"].item())
+        assert status == 0, f"device status {status}"
+        return ev[0].elapsed_time(ev[K]), step_ms, moved
+
+    def parity_step(self, n_units=16, cores=1, time_oracle=False):
+        """One more evicting step, checked against the CPU oracle on a sample of units in this very launch
+        shape.  With time_oracle the oracle is also timed on ALL units (all cores, then one thread)."""
+        from oracle import compare, oracle
+        wl, kd = self.wl, self.kd
+        U, N = wl.units, wl.budget
+        units = np.unique(np.linspace(0, U - 1, n_units).astype(int))
+        sel = torch.as_tensor(units, device=self.dev)
+        nk, nv = self.stream.next_block()
+        timing = None
+        if time_oracle:
+            pre_k, pre_v = bits(self.k_cache), bits(self.v_cache)
+            if self.slots:
+                pos_t, next_pos = kd.positions()
+                pre_pos = pos_t.cpu().numpy().astype(np.int64)
+
+            def run_oracle(threads):
+                if self.slots:
+                    return oracle.evict_units_bf16_slots(pre_k, pre_v, pre_pos, N, next_pos, bits(nk), bits(nv), N, n_threads=threads)
+                return oracle.evict_units_bf16(pre_k, pre_v, N, bits(nk), bits(nv), N, n_threads=threads)
+            times, used = [], 1
+            for rep in range(3):
+                t0 = time.perf_counter()
+                out = run_oracle(cores)
+                times.append(time.perf_counter() - t0)
+                used = out["threads"]
+                if sum(times) > 12:
+                    break
+            t0 = time.perf_counter()
+            run_oracle(1)
+            single = time.perf_counter() - t0
+            timing = {"value": 1.0 / float(np.mean(times)), "unit": UNIT, "cores": used, "kind": "oracle",
+                      "sample": f"{len(times)} evicting step(s), all {U} units, std::thread over units",
+                      "single_thread_value": 1.0 / single, "single_thread_sample": f"1 evicting step, all {U} units, 1 thread",
+                      "sched_getaffinity": cores, "hardware_concurrency": os.cpu_count()}
+            pre_k, pre_v = pre_k[units], pre_v[units]
+            if self.slots:
+                pre_pos = pre_pos[units]
+        else:
+            pre_k, pre_v = bits(self.k_cache[sel]), bits(self.v_cache[sel])
+            if self.slots:
+                pos_t, next_pos = kd.positions()
+                pre_pos = pos_t[sel].cpu().numpy().astype(np.int64)
+        self.step((nk, nv))
+        torch.cuda.synchronize()
+        sc = kd.scratch()
+        scores, kept = sc["scores"][sel].cpu().numpy(), sc["kept_idx"][sel].cpu().numpy()
+        if self.slots:
+            rep = compare.check_step_slots(pre_k, pre_v, pre_pos, next_pos, N, bits(nk[sel]), bits(nv[sel]), N,
+                                           bits(self.k_cache[sel]), bits(self.v_cache[sel]), scores, kept,
+                                           kd.positions()[0][sel].cpu().numpy(), n_threads=cores)
+        else:
+            rep = compare.check_step(pre_k, pre_v, N, bits(nk[sel]), bits(nv[sel]), N, bits(self.k_cache[sel]),
+                                     bits(self.v_cache[sel]), scores, kept, n_threads=cores)
+        par = {"parity_units_checked": rep["units"], "max_score_err_over_tol": rep["max_score_err_over_tol"],
+               "max_plain_rel_score_err": rep["max_plain_rel"],
+               "max_plain_rel_score_err_all_tokens": rep["max_plain_rel_all_tokens"],
+               "frac_tokens_with_abs_score_below_1e-2": rep["frac_tokens_below_floor"]}
+        return par, timing
+
+    def close(self):
+        self.kd.close()
+        del self.k_cache, self.v_cache, self.stream
+        torch.cuda.empty_cache()
+
+
+def roofline_of(run, moved, step_ms, workload, compaction):
+    from paper_2504_15364_b200 import binding  # noqa: F401
+    peak, peak_src = measured_peak()
+    a_step = algorithmic_bytes(run.wl, moved, run.slots)
+    kern_ms = float(step_ms.mean())
+    achieved = a_step / (kern_ms * 1e-3) / 1e9
+    return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": NCU_TRAFFIC_BYTES.get((workload, compaction)), "peak_source": peak_src,
+            "kernel": ("slot_evict_kernel" if run.slots else "fused_evict_kernel") if run.fused else "staged chain (4 kernels)",
+            "algorithmic_bytes_per_launch": a_step, "moved_rows_per_unit": moved,
+            "kernel_ms": kern_ms, "kernel_ms_median": float(np.median(step_ms)),
+            "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+
+
 def run_ours(args):
-    from paper_2504_15364_b200 import KeyDiff, binding
+    from paper_2504_15364_b200 import binding
     rank, world, local = kdist.init_from_env()
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback)"
     torch.cuda.set_device(local)
@@ -117,129 +248,84 @@ def run_ours(args):
     path = {"auto": binding.KEYDIFF_PATH_AUTO, "staged": binding.KEYDIFF_PATH_STAGED,
             "fused": binding.KEYDIFF_PATH_FUSED}[args.path]
     K, W = args.steps, args.warmup
-    K2 = 0 if args.no_e2e else min(K, 40)
+    K2 = 0 if args.no_e2e else 40
+    cores = len(os.sched_getaffinity(0))
 
-    stream = synth.KVStream(wl, dev, rank=rank)
-    k_cache = torch.zeros(U, N, d, dtype=torch.bfloat16, device=dev)
-    v_cache = torch.zeros_like(k_cache)
-    slots = args.compaction == "slot_reuse"
-    kd = KeyDiff(wl.n_layers, wl.batch, wl.n_kv_heads, d, N, B, path=path, device=local,
-                 compaction=binding.KEYDIFF_COMPACT_SLOT_REUSE if slots else binding.KEYDIFF_COMPACT_ORDERED)
-    info = kd.launch_info()
-    # fill through the library's append path (C_0 = empty)
-    for _ in range(wl.fill_steps):
-        nk, nv = stream.next_block()
-        kd.evict(k_cache, v_cache, nk, nv)
-    assert kd.len == N
-    blocks = [stream.next_block() for _ in range(W)]
-    torch.cuda.synchronize()
-
-    for i in range(W):
-        kd.evict(k_cache, v_cache, *blocks[i])
-    torch.cuda.synchronize()
-
-    # ---- CPU baseline (the oracle as it stands) + a parity check of this very launch shape, taken right after
-    # the warm-up steps, i.e. early in the workload's own stream (the timed steps below may run past its end)
-    cpu = None
-    if not args.no_cpu and rank == 0:
-        from oracle import compare, oracle
-        nk, nv = stream.next_block()
-        pre_k, pre_v = bits(k_cache), bits(v_cache)
-        if slots:
-            pos_t, next_pos = kd.positions()
-            pre_pos = pos_t.cpu().numpy().astype(np.int64)
-        cores = len(os.sched_getaffinity(0))
-        times, used = [], 1
-        for rep in range(3):
-            t0 = time.perf_counter()
-            if slots:
-                out = oracle.evict_units_bf16_slots(pre_k, pre_v, pre_pos, N, next_pos, bits(nk), bits(nv), N, n_threads=cores)
-            else:
-                out = oracle.evict_units_bf16(pre_k, pre_v, N, bits(nk), bits(nv), N, n_threads=cores)
-            times.append(time.perf_counter() - t0)
-            used = out["threads"]
-            if sum(times) > 12:
-                break
-        cpu = {"value": 1.0 / float(np.mean(times)), "unit": UNIT, "cores": used, "kind": "oracle",
-               "sample": f"{len(times)} evicting step(s), all {U} units, std::thread over units"}
-        kd.evict(k_cache, v_cache, nk, nv)
-        torch.cuda.synchronize()
-        sc = kd.scratch()
-        units = np.unique(np.linspace(0, U - 1, 16).astype(int))
-        if slots:
-            rep = compare.check_step_slots(pre_k, pre_v, pre_pos, next_pos, N, bits(nk), bits(nv), N, bits(k_cache), bits(v_cache),
-                                           sc["scores"].cpu().numpy(), sc["kept_idx"].cpu().numpy(),
-                                           kd.positions()[0].cpu().numpy(), units=units, n_threads=cores)
-        else:
-            rep = compare.check_step(pre_k, pre_v, N, bits(nk), bits(nv), N, bits(k_cache), bits(v_cache),
-                                     sc["scores"].cpu().numpy(), sc["kept_idx"].cpu().numpy(), units=units, n_threads=cores)
-        cpu["parity_units_checked"] = rep["units"]
-        cpu["max_score_err_over_tol"] = rep["max_score_err_over_tol"]
-        cpu["max_plain_rel_score_err"] = rep["max_plain_rel"]
-
-    blocks += [stream.next_block() for _ in range(K)]
-    torch.cuda.synchronize()
-    moved0 = kd.moved_rows()
-
-    st = torch.cuda.current_stream(dev)
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(K + 1)]
+    run = Run(wl, args.compaction, path, dev, rank)
+    info = run.info
     sampler = ClockSampler(local)
-    kdist.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    ev[0].record(st)
-    for i in range(K):
-        kd.evict(k_cache, v_cache, *blocks[W + i])
-        ev[i + 1].record(st)
-    torch.cuda.synchronize()
-    sampler.stop_flag = True
-    kdist.barrier()
-    sampler.join()
-    total_ms = ev[0].elapsed_time(ev[K])
-    step_ms = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(K)])
-    moved = (kd.moved_rows() - moved0) / K / U
-    status = int(kd.scratch()["status"].item())
-    assert status == 0, f"device status {status}"
-
+    total_ms, step_ms, moved = run.timed(K, W, sampler)
     total_ms_max = kdist.max_over_ranks(total_ms, dev)
     steps_total = kdist.sum_over_ranks(K, dev)
     value = steps_total / (total_ms_max * 1e-3)
 
+    # ---- CPU baseline (the oracle as it stands) + a parity check in this very launch shape, taken AFTER the timed
+    # steps, i.e. at the far end of the stream
+    cpu = None
+    if not args.no_cpu and rank == 0:
+        par, cpu = run.parity_step(16, cores, time_oracle=True)
+        cpu.update(par)
+
     # ---- end to end: block from pinned host memory, kept-index list + status read back
     e2e = None
     if K2:
-        host_blocks = [tuple(t.cpu().pin_memory() for t in stream.next_block()) for _ in range(K2 + 2)]
+        kd, stream = run.kd, run.stream
+        st = torch.cuda.current_stream(dev)
+        host_blocks = [tuple(t.cpu().pin_memory() for t in stream.next_block()) for _ in range(2 * K2 + 4)]
         kept_h = torch.empty(U, N, dtype=torch.int32).pin_memory()
         status_h = torch.zeros(1, dtype=torch.int32).pin_memory()
-        for i in range(2):
-            kd.evict_host(k_cache, v_cache, *host_blocks[i], kept_h, status_h)
+        for i in range(4):   # staging buffers, copy stream and events are created by the first call
+            kd.evict_host(run.k_cache, run.v_cache, *host_blocks[i], kept_h, status_h)
         kdist.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(st)
         for i in range(K2):
-            kd.evict_host(k_cache, v_cache, *host_blocks[2 + i], kept_h, status_h)
+            kd.evict_host(run.k_cache, run.v_cache, *host_blocks[4 + i], kept_h, status_h)
         e1.record(st)
         torch.cuda.synchronize()
         kdist.barrier()
         e2e_ms = kdist.max_over_ranks(e0.elapsed_time(e1), dev)
+        # the same calls with the stream synchronised after every step: what a caller sees who needs the kept list
+        # before it can prepare the next block (host wall clock: the wait is part of the figure)
+        t0 = time.perf_counter()
+        for i in range(K2):
+            kd.evict_host(run.k_cache, run.v_cache, *host_blocks[4 + K2 + i], kept_h, status_h)
+            st.synchronize()
+        sync_ms = kdist.max_over_ranks((time.perf_counter() - t0) * 1e3, dev)
+        assert int(status_h.item()) == 0
         e2e = {"value": kdist.sum_over_ranks(K2, dev) / (e2e_ms * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": 2 * U * B * d * 2, "d2h_bytes_per_step": U * N * 4 + 4, "steps": K2}
+               "h2d_bytes_per_step": 2 * U * B * d * 2, "d2h_bytes_per_step": U * N * 4 + 4, "steps": K2,
+               "mode": "pipelined: calls enqueued back to back, one synchronise at the end",
+               "synchronised_each_step": {"value": kdist.sum_over_ranks(K2, dev) / (sync_ms * 1e-3), "unit": UNIT,
+                                          "ms_per_step": sync_ms / K2, "timer": "host wall clock, stream synchronised after every call"}}
+    roof = roofline_of(run, moved, step_ms, args.workload, args.compaction) if rank == 0 else None
+    run.close()
+
+    # ---- the other workloads and the other layout, on fewer steps (rank 0 reports; every rank runs them so that
+    # the ranks stay in step)
+    others = []
+    if not args.headline_only:
+        for name in synth.CONFIG_ORDER:
+            for comp in ("ordered", "slot_reuse"):
+                if name == args.workload and comp == args.compaction:
+                    continue
+                owl = synth.WORKLOADS[name]
+                r = Run(owl, comp, binding.KEYDIFF_PATH_AUTO, dev, rank)
+                o_total, o_step, o_moved = r.timed(args.other_steps, 3)
+                row = {"workload": name, "compaction": comp, "units": owl.units, "budget_N": owl.budget, "block_B": owl.block,
+                       "path": "fused" if r.fused else "staged", "cluster_size": r.info["cluster_size"],
+                       "steps": args.other_steps, "ms_per_step": kdist.max_over_ranks(o_total, dev) / args.other_steps}
+                if rank == 0:
+                    ro = roofline_of(r, o_moved, o_step, name, comp)
+                    row.update({k: ro[k] for k in ("kernel", "algorithmic_bytes_per_launch", "achieved", "frac", "frac_of_nominal_8TBs", "traffic")})
+                    if not args.no_cpu:
+                        row.update(r.parity_step(16, cores)[0])
+                others.append(row)
+                r.close()
 
     if rank != 0:
         return
-    peak, peak_src = measured_peak()
-    a_step = algorithmic_bytes(wl, moved, slots)
-    kern_ms = float(step_ms.mean())
-    achieved = a_step / (kern_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get((args.workload, args.compaction)), "peak_source": peak_src,
-                "kernel": ("slot_evict_kernel" if slots else "fused_evict_kernel") if info["path"] == binding.KEYDIFF_PATH_FUSED
-                          else "staged chain (4 kernels)",
-                "algorithmic_bytes_per_launch": a_step, "moved_rows_per_unit": moved,
-                "kernel_ms": kern_ms, "kernel_ms_median": float(np.median(step_ms)),
-                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
-
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": total_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
@@ -249,25 +335,24 @@ def run_ours(args):
                        "path": "fused" if info["path"] == binding.KEYDIFF_PATH_FUSED else "staged",
                        "cluster_size": info["cluster_size"], "replicas": world, "compaction": args.compaction},
             "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": K * info["launches_per_step"],
-            "roofline": roofline, "cpu_baseline": cpu}
+            "roofline": roof, "cpu_baseline": cpu, "other_workloads": others}
     print(json.dumps(line))
 
 
 def run_reference(args):
-    """The CPU oracle, as it stands, on the host cores: each step scores/selects/gathers a bounded
-    sample of units of the same workload; the rate is scaled to whole steps."""
+    """The CPU oracle, as it stands, on the host cores, through its own std::thread driver over the units:
+    every step scores/selects/gathers up to 256 units of the same workload; the rate is scaled to whole steps."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from oracle import oracle
     wl = synth.WORKLOADS[args.workload]
-    sample_units = min(wl.units, 16)
-    small = synth.scaled(wl, n_layers=1, batch=1, n_kv_heads=sample_units)
+    sample_units = min(wl.units, 256)
+    small = wl if sample_units == wl.units else synth.scaled(wl, n_layers=1, batch=1, n_kv_heads=sample_units)
     k_cache, v_cache, stream = synth.prefilled_cache(small, "cpu")
     kc, vc = bits(k_cache), bits(v_cache)
     cores = len(os.sched_getaffinity(0))
-    K, W = args.steps, args.warmup
-    K = min(K, 20)
+    K, W = min(args.steps, 12), min(args.warmup, 3)
     times, used = [], 1
     for i in range(W + K):
         nk, nv = stream.next_block()
@@ -279,7 +364,8 @@ def run_reference(args):
             times.append(dt)
     per_step = float(np.mean(times)) * wl.units / sample_units
     value = 1.0 / per_step
-    sample = f"{sample_units} of {wl.units} units per step, {K} steps, scaled to whole steps"
+    sample = f"{sample_units} of {wl.units} units per step, {K} steps, std::thread over units" + \
+             ("" if sample_units == wl.units else ", scaled to whole steps")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
             "warmup": W, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -301,6 +387,9 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "staged", "fused"])
     ap.add_argument("--compaction", default="ordered", choices=["ordered", "slot_reuse"],
                     help="layout of the kept rows: token order (the headline configuration) or unordered slot reuse")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="skip the short runs of the other workloads and of the other layout (the other_workloads list)")
+    ap.add_argument("--other-steps", type=int, default=20, help="timed steps of each entry of other_workloads")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

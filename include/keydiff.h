@@ -23,6 +23,16 @@
  *     time.  Distinct ctxs are independent.
  *   - There is no CPU fallback: on a machine without a usable sm_100 device
  *     keydiff_create fails with KEYDIFF_ERR_CUDA / KEYDIFF_ERR_UNSUPPORTED.
+ *   - The environment is read once, by keydiff_create, for three launch-tuning aids (integers; unset =
+ *     automatic): KEYDIFF_CLUSTER_SIZE (CTAs per cluster of the fused kernels, 1..16), KEYDIFF_STAGGER_NS
+ *     and KEYDIFF_LATE_NS (start-up delays between clusters, nanoseconds).  They change launch shapes
+ *     only, never results; no other call looks at the environment.
+ *   - Accuracy of the scores (fp32 storage, fp64 oracle): a score is (mu.k)/(||mu|| ||k||).  The
+ *     dot product is accumulated in double precision above chains of four fp32 products, so its error
+ *     is about 1e-8 of the SIZE OF ITS TERMS, kappa = sum_c |mu_c k_c| / (||mu|| ||k||) <= 1; the norms
+ *     and the division add about 4e-7 RELATIVE to the score.  Hence |e_gpu - e| <~ 4e-7 |e| + 3e-8
+ *     kappa: within 1e-5 relative for |e| >= 1e-2 whatever the data; for a score nearer to zero (a
+ *     cancelling sum) the error is bounded by the size of the terms, not by the score.
  *
  * Tensor layouts (bf16, contiguous, row = token):
  *   k_cache, v_cache : [n_layers][batch][n_kv_heads][budget N][head_dim]
@@ -144,8 +154,11 @@ KEYDIFF_API int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out);
  * Asynchronous: returns after enqueueing.  Host-detectable errors (INVALID_ARG,
  * STATE) enqueue nothing and leave len unchanged.  Device-side anomalies (a bounded
  * wait that expired) are written to the status word (keydiff_get_scratch) and the
- * kernels return normally.  Non-finite keys give an unspecified selection, never a
- * fault.
+ * kernels return normally; the call itself has returned KEYDIFF_OK long before.  A non-zero
+ * status word means that the cache rows, scores and lists of that step (and of every later
+ * step of the ctx: the word is never cleared) are unspecified; restore the caches from a
+ * copy and use a new ctx (keydiff_set_len / keydiff_set_positions).  Non-finite keys give an
+ * unspecified selection, never a fault.
  */
 KEYDIFF_API int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache,
                   const void* new_k, const void* new_v,
@@ -218,12 +231,32 @@ KEYDIFF_API int keydiff_get_scratch(const keydiff_ctx* ctx, const float** scores
  * keydiff_get_positions -- slot reuse only (else KEYDIFF_ERR_STATE): device pointer to pos[U][N] int32,
  * the token position (0-based index in the sequence) held by each of the first len slots, valid once
  * the stream work of the latest step has completed, and the position the next new token will get.
- * keydiff_set_len(len) declares slots 0 .. len-1 to hold tokens 0 .. len-1; keydiff_reset starts a new
- * sequence.  In this mode kept_idx[u][s] (keydiff_get_scratch) is the candidate number slot s now holds
+ * keydiff_set_len(len) declares slots 0 .. len-1 to hold tokens 0 .. len-1 and keydiff_reset starts a new
+ * sequence; both are host-side bookkeeping, and the array itself is rewritten to that identity map only
+ * by the NEXT step (until then it still shows the previous sequence).  keydiff_set_positions writes it
+ * at once.  In this mode kept_idx[u][s] (keydiff_get_scratch) is the candidate number slot s now holds
  * (s itself for a cache row that stayed, len + j for block row j), and the moved-rows counter counts
  * the block rows written.  Either output pointer may be NULL.
  */
 KEYDIFF_API int keydiff_get_positions(const keydiff_ctx* ctx, const int32_t** pos, long long* next_pos);
+
+/*
+ * keydiff_set_positions -- slot reuse only (else KEYDIFF_ERR_STATE): resume from a cache the caller
+ * restored.  With slot reuse the cache is not in token order, so keydiff_set_len (slot s = token s) cannot
+ * describe a cache that has already evicted; this call hands the saved position array back.  (The sliding
+ * window of Sec. 3.2 is defined on these positions, and Eq. block_processing carries the cache, hence
+ * its positions, from block to block.)
+ *   pos_device : device, [U][N] int32 as keydiff_get_positions returned it (rows [0, len) of every unit
+ *                are used), copied into the ctx on `stream`; NULL = the identity map (slot s = token s)
+ *   len        : cached tokens per unit, 0 <= len <= N
+ *   next_pos   : position the next new token gets, len <= next_pos < 2^31; every stored position must
+ *                be below it (not checked)
+ * The running anchor sum is rebuilt by the next evicting step.  Asynchronous on `stream`; later steps
+ * must be enqueued on the same stream or ordered after it.  Errors: INVALID_ARG, STATE (not slot reuse,
+ * or the ctx's device is not current), CUDA.
+ */
+KEYDIFF_API int keydiff_set_positions(keydiff_ctx* ctx, const int32_t* pos_device, int32_t len, long long next_pos,
+                                      void* stream);
 
 /*
  * keydiff_get_moved_rows -- device pointer to a 64-bit counter: the number of kept rows (per
@@ -262,9 +295,10 @@ KEYDIFF_API int keydiff_get_launch_info(const keydiff_ctx* ctx, int32_t* path, i
  * B=128; about 2100 units at N=512, B=128) and len+block_B must not exceed 51200; otherwise the call
  * returns KEYDIFF_ERR_TOO_LARGE and enqueues nothing.
  *
- * Set-up: the first call on each device looks up the array's device address
- * (cudaGetSymbolAddress) and sets one kernel attribute; the device must be current.  Make that
- * first call before starting any stream capture.  Later calls do no set-up.
+ * Set-up: the first call on each device -- whatever it does, an append-only step included -- looks up
+ * the array's device address (cudaGetSymbolAddress) and sets one kernel attribute before it enqueues
+ * anything; the device that holds the tensors must be current (checked for k_cache: KEYDIFF_ERR_STATE).
+ * Make that first call before starting any stream capture.  Later calls do no set-up.
  *
  * Sharing: every call on a device uses the same array, and the array keeps whatever the previous
  * call left in it (the call clears the one counter that has to start at zero).  Two calls whose
@@ -274,6 +308,25 @@ KEYDIFF_API int keydiff_get_launch_info(const keydiff_ctx* ctx, int32_t* path, i
 KEYDIFF_API int keydiff_evict_static(void* k_cache, void* v_cache, const void* new_k, const void* new_v,
                                      int32_t len, int32_t budget_N, int32_t block_B, int32_t n_units,
                                      int32_t head_dim, float eps, void* stream);
+
+/*
+ * keydiff_selftest_bounded_wait -- failure-detection self test (the paper has no counterpart).  Every
+ * wait of the kernels on a copy in flight is bounded; when one runs out, the kernel writes
+ * KEYDIFF_ERR_TIMEOUT to its status word and still returns normally.  This call shows that behaviour
+ * without disturbing anything: it launches one small CTA on `stream` whose threads wait, through the same
+ * wait routine and with a limit of `polls` polls (1..4096), on a barrier that nothing ever completes.
+ * After the stream work has completed, *status_device (device, int32, caller-owned, zeroed by the
+ * caller) holds KEYDIFF_ERR_TIMEOUT.  Errors: INVALID_ARG, CUDA.
+ */
+KEYDIFF_API int keydiff_selftest_bounded_wait(int32_t* status_device, int32_t polls, void* stream);
+
+/*
+ * keydiff_debug_fail_alloc -- test hook: the nth device allocation (1-based) that the next keydiff_create
+ * makes on this process fails once, as if the device were out of memory; keydiff_create must then
+ * release what it had allocated and return KEYDIFF_ERR_ALLOC.  0 disarms.  The hook is disarmed when
+ * keydiff_create returns.  Not thread-safe.
+ */
+KEYDIFF_API int keydiff_debug_fail_alloc(int32_t nth);
 
 /* Text of a status code; never NULL. */
 KEYDIFF_API const char* keydiff_strerror(int code);

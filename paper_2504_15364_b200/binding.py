@@ -27,6 +27,7 @@ KEYDIFF_COMPACT_ORDERED, KEYDIFF_COMPACT_SLOT_REUSE = 0, 1
 EXPORTS = ["keydiff_create", "keydiff_evict", "keydiff_evict_host", "keydiff_destroy", "keydiff_reset",
            "keydiff_get_len", "keydiff_set_len", "keydiff_get_scratch", "keydiff_get_moved_rows",
            "keydiff_get_launch_info", "keydiff_evict_static", "keydiff_set_incremental", "keydiff_get_positions",
+           "keydiff_set_positions", "keydiff_selftest_bounded_wait", "keydiff_debug_fail_alloc",
            "keydiff_strerror", "keydiff_last_cuda_error"]
 
 
@@ -69,6 +70,9 @@ def load_library() -> ctypes.CDLL:
     lib.keydiff_get_scratch.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp)]
     lib.keydiff_get_moved_rows.argtypes = [vp, ctypes.POINTER(vp)]
     lib.keydiff_get_positions.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_longlong)]
+    lib.keydiff_set_positions.argtypes = [vp, vp, i32, ctypes.c_longlong, vp]
+    lib.keydiff_selftest_bounded_wait.argtypes = [vp, i32, vp]
+    lib.keydiff_debug_fail_alloc.argtypes = [i32]
     lib.keydiff_get_launch_info.argtypes = [vp, i32p, i32p, i32p]
     lib.keydiff_evict_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, ctypes.c_float, vp]
     lib.keydiff_strerror.argtypes = [ctypes.c_int]
@@ -189,6 +193,15 @@ class KeyDiff:
         _check(self._lib.keydiff_get_positions(self._ctx, ctypes.byref(p), ctypes.byref(nxt)))
         return torch.as_tensor(_DevArray(p.value, (self.units, self.budget), "<i4"), device=self.device), nxt.value
 
+    def set_positions(self, pos, length: int, next_pos: int, stream: torch.cuda.Stream | None = None):
+        """``keydiff_set_positions`` (slot reuse only): resume from a restored cache whose slot -> token position
+        map is ``pos`` (int32 CUDA tensor [U, N]; None = identity)."""
+        if pos is not None:
+            if pos.dtype != torch.int32 or not pos.is_cuda or not pos.is_contiguous() or pos.numel() != self.units * self.budget:
+                raise KeyDiffError(KEYDIFF_ERR_INVALID_ARG, "pos: need a contiguous int32 CUDA tensor [U, N]")
+        st = (stream or torch.cuda.current_stream(self.device)).cuda_stream
+        _check(self._lib.keydiff_set_positions(self._ctx, pos.data_ptr() if pos is not None else None, length, next_pos, st))
+
     def moved_rows(self) -> int:
         """Cumulative count of kept rows that changed position (synchronises the device)."""
         p = ctypes.c_void_p()
@@ -229,6 +242,24 @@ def evict_static(k_cache, v_cache, new_k, new_v, length: int, stream: torch.cuda
             raise KeyDiffError(KEYDIFF_ERR_INVALID_ARG, "need contiguous bf16 CUDA tensors")
     assert v_cache.shape == k_cache.shape and new_k.shape == (U, B, d) and new_v.shape == (U, B, d)
     st = (stream or torch.cuda.current_stream(k_cache.device)).cuda_stream
-    _check(lib.keydiff_evict_static(k_cache.data_ptr(), v_cache.data_ptr(), new_k.data_ptr(), new_v.data_ptr(),
-                                    length, N, B, U, d, eps, st))
+    with torch.cuda.device(k_cache.device):   # the library looks the scratch up for the current device
+        _check(lib.keydiff_evict_static(k_cache.data_ptr(), v_cache.data_ptr(), new_k.data_ptr(), new_v.data_ptr(),
+                                        length, N, B, U, d, eps, st))
     return min(N, length + B)
+
+
+def selftest_bounded_wait(polls: int = 1000, device=None) -> int:
+    """``keydiff_selftest_bounded_wait``: runs the library's bounded wait on a barrier nothing completes and
+    returns the status word it leaves (KEYDIFF_ERR_TIMEOUT when failure detection works)."""
+    lib = load_library()
+    dev = torch.device("cuda", torch.cuda.current_device() if device is None else device)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib.keydiff_selftest_bounded_wait(status.data_ptr(), polls, torch.cuda.current_stream(dev).cuda_stream))
+        torch.cuda.synchronize(dev)
+    return int(status.item())
+
+
+def debug_fail_alloc(nth: int):
+    """``keydiff_debug_fail_alloc``: make the nth device allocation of the next ``keydiff_create`` fail."""
+    _check(load_library().keydiff_debug_fail_alloc(nth))

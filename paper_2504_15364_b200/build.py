@@ -22,17 +22,23 @@ def _stale() -> bool:
     return any(p.stat().st_mtime > t for p in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> Path:
-    """Compile libkeydiff.so in-tree if missing or older than its sources."""
-    if not force and not _stale():
-        return LIB
+STAMPS_LIB = PKG / "libkeydiff_stamps.so"   # diagnostic build: fused kernel with per-phase timers (phase_times.py)
+
+
+def build_library(force: bool = False, verbose: bool = False, phase_stamps: bool = False) -> Path:
+    """Compile libkeydiff.so in-tree if missing or older than its sources.  phase_stamps=True builds the
+    diagnostic variant libkeydiff_stamps.so instead (-DKEYDIFF_PHASE_STAMPS: the fused kernel times its phases)."""
+    out = STAMPS_LIB if phase_stamps else LIB
+    if not force and not phase_stamps and not _stale():
+        return out
     nvcc = os.environ.get("NVCC", "nvcc")
-    tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
-    cmd = [nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), *map(str, SOURCES), "-o", str(tmp)]
+    tmp = out.with_suffix(f".{os.getpid()}.tmp")
+    cmd = [nvcc, *NVCC_FLAGS, *(["-DKEYDIFF_PHASE_STAMPS"] if phase_stamps else []), *(["-Xptxas", "-v"] if verbose else []),
+           *map(str, SOURCES), "-o", str(tmp)]
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":
-    print(build_library(force=True, verbose="-v" in sys.argv))
+    print(build_library(force=True, verbose="-v" in sys.argv, phase_stamps="--phase-stamps" in sys.argv))

@@ -44,11 +44,25 @@ __device__ __forceinline__ float row_sumsq(const float (&x)[16]) {
     return group_sum(s0 + s1);
 }
 
+// mu.k over the row group.  Products and chains of four of them are fp32 (a product of a bf16 value and an
+// fp32 value rounds at the size of that one term); everything above them -- the four chains of a lane and
+// the eight lanes of the group -- is added in double precision, because a cosine near zero is a sum of
+// terms that cancel and fp32 partial sums of the size of the terms would decide its last digits.
+__device__ __forceinline__ double group_sum(double v) {
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    v += __shfl_xor_sync(0xffffffffu, v, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 4);
+    return v;
+}
 __device__ __forceinline__ float row_dot(const float (&x)[16], const float (&w)[16]) {
-    float s0 = 0.f, s1 = 0.f;
+    float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int j = 0; j < 8; ++j) { s0 = fmaf(x[j], w[j], s0); s1 = fmaf(x[8 + j], w[8 + j], s1); }
-    return group_sum(s0 + s1);
+    for (int j = 0; j < 4; ++j) {
+        c[0] = fmaf(x[j], w[j], c[0]); c[1] = fmaf(x[4 + j], w[4 + j], c[1]);
+        c[2] = fmaf(x[8 + j], w[8 + j], c[2]); c[3] = fmaf(x[12 + j], w[12 + j], c[3]);
+    }
+    const double lane = (static_cast<double>(c[0]) + static_cast<double>(c[1])) + (static_cast<double>(c[2]) + static_cast<double>(c[3]));
+    return static_cast<float>(group_sum(lane));
 }
 
 // App. B.1, second expression, then the eviction score e = -s with -0 mapped to +0.

@@ -52,12 +52,13 @@ constexpr int kCandCap = kFusedThreads;                 // exact-rank stage hand
 constexpr int kMaxCluster = 16;
 constexpr int kFastKeys = 17;                           // fast select: keys per thread held in registers (n <= 8704)
 constexpr int kFastCandCap = 192;                       // fast select: keys of the threshold bin ranked exactly
+constexpr int kReduceBytes = 28 * 1024;   // scratch the dead key table lends: staged row terms (16 KB), quarter sums, lists
 constexpr int kSmemLimit = 232448;                      // opt-in shared memory per CTA on sm_100
 constexpr int kErrTimeout = -6;                         // KEYDIFF_ERR_TIMEOUT
 constexpr uint32_t kWaitSpins = 1u << 24;               // bound of every mbarrier wait
 
 struct FusedLayout {
-    int rows, keys, work, xchg, sel, mu, mbar, misc, total;
+    int rows, keys, work, xchg, bitmap, sel, mu, mbar, misc, total;
 };
 
 // Shared-memory carve-up for a slice with `smem_rows` resident rows, a key table of nkeys
@@ -67,11 +68,12 @@ __host__ __device__ inline FusedLayout fused_layout(int smem_rows, int nkeys, in
     int off = 0;
     auto take = [&off](int bytes) { const int o = off; off += (bytes + 127) & ~127; return o; };
     L.rows = take(smem_rows * kRowBytes);
-    L.keys = take(nkeys * 4 > kBins * 4 ? nkeys * 4 : kBins * 4);   // also 8 KB of reduction scratch while the table is dead
+    L.keys = take(nkeys * 4 > kReduceBytes ? nkeys * 4 : kReduceBytes);   // also the reduction scratch while the table is dead
     L.work = take(kBins * 4);   // warp-reduction scratch / histogram / destination table (never live together)
-    L.xchg = take(C * kHeadDim * 4 > 2 * kCandCap * 4 ? C * kHeadDim * 4 : 2 * kCandCap * 4);   // anchor partials [C][128] / candidates
+    L.xchg = take(2 * kCandCap * 4 + C * kHeadDim * 8);   // candidates of the threshold bin | [C][128] doubles pushed by the peers
+    L.bitmap = take(2 * ((nkeys + 31) / 32) * 4);   // evicted-token bitmap, evicted-before count of every word
     L.sel = take(static_cast<int>(sizeof(SelectSmem)));
-    L.mu = take(kHeadDim * 4);
+    L.mu = take(2 * kHeadDim * 4);   // this unit's anchor and the next unit's
     L.mbar = take(kMaxTiles * 8);
     L.misc = take(128);
     L.total = off;
@@ -93,7 +95,7 @@ struct FusedParams {
     // running anchor (see the kernel): sum of k/||k|| over the cached rows as of the previous step
     // = anchor_in[u][c] + sum over CTA ranks r of anchor_delta[u][r][c]; this step writes anchor_out and
     // new deltas
-    const double* anchor_in; double* anchor_out; float* anchor_delta;
+    const double* anchor_in; double* anchor_out; double* anchor_delta;
     int raw_anchor;     // 1: the anchor is the mean of the keys themselves (Sec. 3.2), 0: of the normalised keys
     int window;         // w most recent tokens that are never evicted (Sec. 3.2, sliding window)
     int32_t* kept_mirror;   // optional second destination of the kept-index list (device alias of pinned host memory)
@@ -135,12 +137,50 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
 }
 
-// Bounded wait; returns false (and records the timeout) if the phase never completed.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status) {
-    for (uint32_t spin = 0; spin < kWaitSpins; ++spin)
+// Optional per-phase timing (build with -DKEYDIFF_PHASE_STAMPS, see build.py --phase-stamps): thread 0 of every CTA
+// adds the time since its previous stamp to the phase's total; at the end of the kernel the totals go to
+// g_phase_ns[CTA][phase], which keydiff_debug_phase_ns reads.  Without the macro nothing of this is compiled.
+constexpr int kMaxPhases = 16;
+constexpr int kMaxStampCtas = 2368;   // 148 SMs x 16
+#ifdef KEYDIFF_PHASE_STAMPS
+__device__ unsigned long long g_phase_ns[kMaxStampCtas][kMaxPhases];
+#define KD_STAMP_DECL __shared__ unsigned long long stamp_sh[kMaxPhases + 1]; \
+    if (threadIdx.x == 0) { for (int i_ = 0; i_ < kMaxPhases; ++i_) stamp_sh[i_] = 0; stamp_sh[kMaxPhases] = global_timer_ns(); }
+#define KD_STAMP(id) do { if (threadIdx.x == 0) { const unsigned long long now_ = global_timer_ns(); \
+    stamp_sh[id] += now_ - stamp_sh[kMaxPhases]; stamp_sh[kMaxPhases] = now_; } } while (0)
+#define KD_STAMP_FLUSH do { if (threadIdx.x == 0 && blockIdx.x < kMaxStampCtas) \
+    for (int i_ = 0; i_ < kMaxPhases; ++i_) atomicAdd(&g_phase_ns[blockIdx.x][i_], stamp_sh[i_]); } while (0)
+#else
+#define KD_STAMP_DECL
+#define KD_STAMP(id) do {} while (0)
+#define KD_STAMP_FLUSH do {} while (0)
+#endif
+
+// Bounded wait; returns false if the phase never completed.  The first wait that runs out records
+// KEYDIFF_ERR_TIMEOUT in the status word; while the status word is non-zero every other wait gives up after
+// a thousand polls instead of waiting its full length again, so a kernel in which one copy never lands still
+// ends within milliseconds.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t* status, uint32_t limit = kWaitSpins) {
+    for (uint32_t spin = 0; spin < limit; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 1023u) == 1023u && *reinterpret_cast<volatile int32_t*>(status) != 0) return false;
+    }
     atomicExch(status, kErrTimeout);
     return false;
+}
+
+// Failure-detection self test: every thread waits, with a limit of `polls` polls, on an mbarrier that nothing
+// ever completes (no arrival, no copy).  The waits run out, the status word receives KEYDIFF_ERR_TIMEOUT and
+// the kernel returns normally: exactly what a product kernel does when a copy never lands.
+__global__ void bounded_wait_selftest_kernel(int32_t* status, uint32_t polls) {
+    __shared__ __align__(8) unsigned long long bar;
+    const uint32_t bar_sa = smem_addr(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(bar_sa, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    mbar_wait(bar_sa, 0u, status, polls);   // phase 0 never completes
 }
 
 // inverse of order_key
@@ -200,11 +240,20 @@ __device__ __forceinline__ float pairs_sumsq(const float2 (&x)[8]) {
     for (int p = 0; p < 4; ++p) { s0 = __ffma2_rn(x[p], x[p], s0); s1 = __ffma2_rn(x[4 + p], x[4 + p], s1); }
     return group_sum((s0.x + s0.y) + (s1.x + s1.y));
 }
-__device__ __forceinline__ float pairs_dot(const float2 (&x)[8], const float2 (&w)[8]) {
-    float2 s0 = make_float2(0.f, 0.f), s1 = s0;
+// mu.k.  Products and chains of four of them are fp32: such a chain rounds at the size of a few terms, and 32
+// chains with independent roundings leave about 1e-8 of the size of the terms.  Everything above the chains --
+// the four chains of a lane, the eight lanes of the row group -- is added in double precision: a cosine near
+// zero is a cancelling sum, and fp32 partial sums of the size of ALL its terms would decide its last digits.
+__device__ __forceinline__ double lane_dot(const float2 (&x)[8], const float2 (&w)[8]) {
+    float2 d0 = make_float2(0.f, 0.f), d1 = d0;
 #pragma unroll
-    for (int p = 0; p < 4; ++p) { s0 = __ffma2_rn(x[p], w[p], s0); s1 = __ffma2_rn(x[4 + p], w[4 + p], s1); }
-    return group_sum((s0.x + s0.y) + (s1.x + s1.y));
+    for (int p = 0; p < 4; ++p) { d0 = __ffma2_rn(x[p], w[p], d0); d1 = __ffma2_rn(x[4 + p], w[4 + p], d1); }
+    return (static_cast<double>(d0.x) + static_cast<double>(d0.y)) + (static_cast<double>(d1.x) + static_cast<double>(d1.y));
+}
+// This lane's 16 anchor channels as fp32 pairs: w[q] = channels lane_channel(t, 2q), lane_channel(t, 2q + 1).
+__device__ __forceinline__ void load_anchor(const float* mu, int t, float2 (&w)[8]) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) w[q] = *reinterpret_cast<const float2*>(&mu[lane_channel(t, 2 * q)]);
 }
 // Step a1 for one row: returns ||k||; adds k / max(||k||, eps) into acc when the row is valid.
 // 1/max(r, eps) = min(1/r, 1/eps); the reciprocal square root and the square root are the
@@ -220,56 +269,86 @@ __device__ __forceinline__ float row_a1(const uint4& a, const uint4& b, bool val
     for (int p = 0; p < 8; ++p) acc[p] = __ffma2_rn(x[p], inv2, acc[p]);
     return approx_sqrt(ss);
 }
-// Steps a1 + a2 for one row when the anchor is known beforehand: norm and dot product in one pass.
-__device__ __forceinline__ uint32_t row_score(const uint4& a, const uint4& b, const float2 (&w)[8], float m, float eps) {
+// One lane's share of ||k||^2 (fp32: the norm only enters the score as a factor) and of mu.k (double), no
+// exchange between lanes yet.
+__device__ __forceinline__ void lane_sumsq_dot(const uint4& a, const uint4& b, const float2 (&w)[8], float& ss, double& dot) {
     float2 x[8];
     unpack_pairs(a, b, x);
-    const float r = approx_sqrt(pairs_sumsq(x));
-    const float dot = pairs_dot(x, w);
-    const float e = -(dot * approx_rcp(fmaxf(m * r, eps)));
-    return order_key(e == 0.f ? 0.f : e);
-}
-// One lane's share of ||k||^2 and of mu.k (no exchange between lanes yet).
-__device__ __forceinline__ void lane_sumsq_dot(const uint4& a, const uint4& b, const float2 (&w)[8], float& ss, float& dot) {
-    float2 x[8];
-    unpack_pairs(a, b, x);
-    float2 s0 = make_float2(0.f, 0.f), s1 = s0, d0 = s0, d1 = s0;
+    float2 s0 = make_float2(0.f, 0.f), s1 = s0;
 #pragma unroll
-    for (int p = 0; p < 4; ++p) {
-        s0 = __ffma2_rn(x[p], x[p], s0); s1 = __ffma2_rn(x[4 + p], x[4 + p], s1);
-        d0 = __ffma2_rn(x[p], w[p], d0); d1 = __ffma2_rn(x[4 + p], w[4 + p], d1);
-    }
+    for (int p = 0; p < 4; ++p) { s0 = __ffma2_rn(x[p], x[p], s0); s1 = __ffma2_rn(x[4 + p], x[4 + p], s1); }
     ss = (s0.x + s0.y) + (s1.x + s1.y);
-    dot = (d0.x + d0.y) + (d1.x + d1.y);
+    dot = lane_dot(x, w);
 }
-// Eight values per lane, each to be summed over the 8 lanes of a row group: a butterfly that halves
-// the values it carries at every step (4 + 2 + 1 shuffles instead of 8 x 3).  Lane t (0..7 within the
-// group) returns the group's sum of v[t].
-__device__ __forceinline__ float group_sum8(const float (&v)[8], int t) {
-    float r4[4], r2[2];
-    const bool h4 = t & 4, h2 = t & 2, h1 = t & 1;
+// Four values per lane, each to be summed over the 8 lanes of a row group: a butterfly that halves the
+// values it carries (2 + 1 + 1 exchanges instead of 4 x 3).  Lane t (0..7 within the group) returns the
+// group's sum of v[t >> 1].
+template <typename T>
+__device__ __forceinline__ T group_sum4(const T (&v)[4], int t) {
+    const bool h4 = t & 4, h2 = t & 2;
+    T r2[2];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) r4[i] = (h4 ? v[i + 4] : v[i]) + __shfl_xor_sync(0xffffffffu, h4 ? v[i] : v[i + 4], 4);
-#pragma unroll
-    for (int i = 0; i < 2; ++i) r2[i] = (h2 ? r4[i + 2] : r4[i]) + __shfl_xor_sync(0xffffffffu, h2 ? r4[i] : r4[i + 2], 2);
-    return (h1 ? r2[1] : r2[0]) + __shfl_xor_sync(0xffffffffu, h1 ? r2[0] : r2[1], 1);
+    for (int i = 0; i < 2; ++i) r2[i] = (h4 ? v[i + 2] : v[i]) + __shfl_xor_sync(0xffffffffu, h4 ? v[i] : v[i + 2], 4);
+    const T r1 = (h2 ? r2[1] : r2[0]) + __shfl_xor_sync(0xffffffffu, h2 ? r2[0] : r2[1], 2);
+    return r1 + __shfl_xor_sync(0xffffffffu, r1, 1);
 }
-// Keys of four rows of a row group from the lanes' shares v[2i] = ||k_i||^2, v[2i+1] = mu.k_i: after
-// the butterfly lane 2i holds row i's squared norm and fetches its dot product from lane 2i+1.
-// Returns row (t >> 1)'s key in the even lanes (odd lanes: unspecified).
-__device__ __forceinline__ uint32_t score4(const float (&v)[8], int t, float m, float eps) {
-    const float mine = group_sum8(v, t);
-    const float dot = __shfl_xor_sync(0xffffffffu, mine, 1);
-    const float e = -(dot * approx_rcp(fmaxf(m * approx_sqrt(mine), eps)));
+// Keys of four rows of a row group from the lanes' shares ss[i] of ||k_i||^2 and dot[i] of mu.k_i: lane t
+// returns row (t >> 1)'s key.
+__device__ __forceinline__ uint32_t score4(const float (&ss)[4], const double (&dot)[4], int t, float m, float eps) {
+    const float r2 = group_sum4(ss, t);
+    const float d = static_cast<float>(group_sum4(dot, t));
+    const float e = -(d * approx_rcp(fmaxf(m * approx_sqrt(r2), eps)));
     return order_key(e == 0.f ? 0.f : e);
 }
 // Step a2 for one row: orderable key of e = -(mu.k)/max(||mu|| ||k||, eps), -0 mapped to +0.
 __device__ __forceinline__ uint32_t row_a2(const uint4& a, const uint4& b, const float2 (&w)[8], float m, float r, float eps) {
     float2 x[8];
     unpack_pairs(a, b, x);
-    const float dot = pairs_dot(x, w);
+    const float dot = static_cast<float>(group_sum(lane_dot(x, w)));
     const float e = -(dot * approx_rcp(fmaxf(m * r, eps)));
     return order_key(e == 0.f ? 0.f : e);
+}
+
+// Sum over the CTA of every thread's 16 channel accumulators (fp32 sums over a few rows each), carried in double
+// from here on: an anchor sum over thousands of unit vectors cancels when the keys point in many directions, and
+// fp32 partial sums of its size would limit the anchor's accuracy (hence every score's) to about 1e-7 / ||mu||.
+// Returns channel tid's sum in threads tid < 128 (0 elsewhere).  scratch: half * 8 * 128 doubles, half = 1
+// (two rounds of eight warps) or 2 (one round); ends after a CTA barrier only when the caller adds one.
+template <int kHalf>
+__device__ __forceinline__ double cta_channel_sum(const double (&v)[16], double* scratch, int tid) {
+    const int lane = tid & 31, warp = tid >> 5, t = tid & 7;
+    double r[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        double x = v[j];
+        x += __shfl_xor_sync(0xffffffffu, x, 8);
+        x += __shfl_xor_sync(0xffffffffu, x, 16);
+        r[j] = x;
+    }
+    double s = 0.0;
+    constexpr int kWarpsPerRound = 8 * kHalf;
+#pragma unroll 1
+    for (int w0 = 0; w0 < kFusedWarps; w0 += kWarpsPerRound) {
+        if (w0 > 0) __syncthreads();   // the previous round's values have been read
+        if (lane < 8 && warp >= w0 && warp < w0 + kWarpsPerRound) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                *reinterpret_cast<double2*>(&scratch[(warp - w0) * kHeadDim + lane_channel(t, 2 * q)]) = make_double2(r[2 * q], r[2 * q + 1]);
+        }
+        __syncthreads();
+        if (tid < kHeadDim) {
+#pragma unroll
+            for (int w = 0; w < kWarpsPerRound; ++w) s += scratch[w * kHeadDim + tid];
+        }
+    }
+    return s;
+}
+__device__ __forceinline__ void widen_acc(const float2 (&acc)[8], double (&v)[16]) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) { v[2 * q] = static_cast<double>(acc[q].x); v[2 * q + 1] = static_cast<double>(acc[q].y); }
+}
+__device__ __forceinline__ void st_cluster_f64(uint32_t addr, double v) {
+    asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
 }
 
 // Search in the 2048-bin histogram from the low end, two levels and one CTA barrier: warp w sums bins
@@ -306,6 +385,105 @@ __device__ __forceinline__ int find_crossing(const int* h, int E, int lane, int 
     before += cy;
     if (before + cz >= E) return ((bin + 2) << 16) | before;
     return ((bin + 3) << 16) | (before + cz);
+}
+
+// Selection at the low end of the key table (every thread of the CTA calls; the result is uniform).  Only
+// E = n - N keys go, so thread t keeps the keys of tokens t, t + 512, ... in registers (n <= 8704); the 2048
+// bins are spread over the low end of the unit's own key range, from the smallest key to a bound on the
+// E-th smallest (monotone in the key, which is all selection needs); the tokens under the threshold bin go
+// straight into the bitmap, the bin's own few keys are ranked exactly under (key ascending, index
+// descending) = the reverse of the keep order.  On entry hist and bitmap are zero, misc[0] = 0, misc[1] = n,
+// all visible to the CTA.  Returns true with the evicted tokens' bits set in `bitmap` and misc[1] = the first
+// evicted token (both visible to the CTA), or false when the threshold bin holds more than kFastCandCap
+// keys (many equal scores): the bitmap and misc are then in an unspecified state and the caller takes the
+// full-table route.  cand_key / cand_idx: kFastCandCap entries each.
+__device__ __forceinline__ bool low_end_select(const uint32_t* keys, int n, int E, int* hist, uint32_t* bitmap,
+                                               uint32_t* cand_key, int* cand_idx, SelectSmem& sel, int* misc) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t* wmin = reinterpret_cast<uint32_t*>(sel.hist);          // (sel.hist is radix-select scratch)
+    uint32_t* wmax = reinterpret_cast<uint32_t*>(sel.hist) + kFusedWarps;
+    const int cnt = (n - tid + kFusedThreads - 1) / kFusedThreads;
+    uint32_t kk[kFastKeys];
+#pragma unroll
+    for (int j = 0; j < kFastKeys; ++j) kk[j] = j < cnt ? keys[tid + j * kFusedThreads] : 0xffffffffu;
+    {
+        uint32_t lo = 0xffffffffu, hi = 0u;
+#pragma unroll
+        for (int j = 0; j < kFastKeys; ++j) { lo = min(lo, kk[j]); if (j < cnt) hi = max(hi, kk[j]); }
+        // The E-th smallest key is at most the largest of any E distinct keys.  When at least E
+        // threads hold keys, the thread minima are such keys, so the largest thread minimum bounds
+        // it; otherwise the largest key does.  Keys above the bound share the top bin.
+        const uint32_t cut = (n >= kFusedThreads && E <= kFusedThreads) ? lo : hi;
+        const uint32_t wlo = __reduce_min_sync(0xffffffffu, lo);
+        const uint32_t wcut = __reduce_max_sync(0xffffffffu, cnt > 0 ? cut : 0u);
+        if (lane == 0) { wmin[warp] = wlo; wmax[warp] = wcut; }
+    }
+    __syncthreads();
+    uint32_t kmin, kcut, shift;
+    {
+        const uint32_t lo = lane < kFusedWarps ? wmin[lane] : 0xffffffffu, hi = lane < kFusedWarps ? wmax[lane] : 0u;
+        kmin = __reduce_min_sync(0xffffffffu, lo);
+        kcut = __reduce_max_sync(0xffffffffu, hi);
+        const int bits = 32 - __clz(kcut - kmin);   // significant bits of the range [kmin, kcut]
+        shift = bits > 11 ? bits - 11 : 0;          // (key - kmin) >> shift < 2048 inside the range
+    }
+    // bin of a key: linear in the key over [kmin, kcut] (bins 0..2046), 2047 above; monotone
+    auto bin_of = [kmin, kcut, shift](uint32_t k) { return k <= kcut ? min((k - kmin) >> shift, 2046u) : 2047u; };
+#pragma unroll
+    for (int j = 0; j < kFastKeys; ++j) {
+        // (the top bin holds every key above the bound: the crossing is never there, so it is not counted)
+        const uint32_t b = bin_of(kk[j]);
+        if (j < cnt && b != 2047u) atomicAdd(&hist[b], 1);
+    }
+    __syncthreads();
+    const int packed = find_crossing(hist, E, lane, warp, sel.warp_eq);
+    const uint32_t bstar = static_cast<uint32_t>(packed >> 16);
+    const int need = E - (packed & 0xffff);   // this many keys of the threshold bin go
+    unsigned m_below = 0, m_in = 0;           // bit j: this thread's j-th key is below / inside the bin
+#pragma unroll
+    for (int j = 0; j < kFastKeys; ++j) {
+        const uint32_t b = bin_of(kk[j]);
+        m_below |= (j < cnt && b < bstar) ? 1u << j : 0u;
+        m_in |= (j < cnt && b == bstar) ? 1u << j : 0u;
+    }
+    {
+        int first = n;
+        if (packed >= 0 && (m_below | m_in)) {
+            for (unsigned m = m_below; m; m &= m - 1) {
+                const int i = tid + (__ffs(m) - 1) * kFusedThreads;
+                atomicOr(&bitmap[i >> 5], 1u << (i & 31));
+                first = min(first, i);
+            }
+            for (unsigned m = m_in; m; m &= m - 1) {
+                const int i = tid + (__ffs(m) - 1) * kFusedThreads;
+                const int slot = atomicAdd(&misc[0], 1);
+                if (slot < kFastCandCap) { cand_key[slot] = keys[i]; cand_idx[slot] = i; }
+            }
+        }
+        first = __reduce_min_sync(0xffffffffu, first);   // one shared-memory atomic per warp, not per thread
+        if (lane == 0 && first < n) atomicMin(&misc[1], first);
+    }
+    __syncthreads();
+    const int ncand = misc[0];
+    const bool ok = packed >= 0 && ncand <= kFastCandCap;   // the same in every thread
+    if (ok) {
+        int wfirst = n;
+        for (int c = warp; c < ncand; c += kFusedWarps) {
+            const uint32_t mk = cand_key[c];
+            const int mi = cand_idx[c];
+            int rank = 0;
+            for (int q = lane; q < ncand; q += 32) {
+                const uint32_t ok2 = cand_key[q];
+                rank += (ok2 < mk) || (ok2 == mk && cand_idx[q] > mi);
+            }
+            rank = __reduce_add_sync(0xffffffffu, rank);
+            if (lane == 0 && rank < need) { atomicOr(&bitmap[mi >> 5], 1u << (mi & 31)); wfirst = min(wfirst, mi); }
+        }
+        if (lane == 0 && wfirst < n) atomicMin(&misc[1], wfirst);
+    }
+    // Every thread has read misc[0] by now; whoever runs next (the full-table route resets misc) may write it.
+    __syncthreads();
+    return ok;
 }
 
 // Exact top-N over the whole key table by one CTA (every CTA of the cluster runs it on its own
@@ -414,18 +592,160 @@ __device__ __noinline__ void full_select_plan(const uint32_t* keys, int n, int N
     __syncthreads();
 }
 
+// The anchor's running sum (App. B.1, first expression, carried across steps) is kept so that it cannot drift:
+// EVERY ROW'S TERM IS A FIXED BIT PATTERN -- the fp32 products of the row's bf16 elements and the row's fp32
+// reciprocal norm, both functions of the row alone -- and terms are added and subtracted in double precision.  A
+// row that enters the cache adds exactly what it takes away when it is evicted, and no fp32 partial sum of the
+// size of the anchor appears anywhere (an anchor over keys that point in many directions is a cancelling sum;
+// fp32 partial sums would limit it, and with it every score, to about 1e-7 / ||mu||).
+//
+// row_terms: one row group (8 lanes, lane t holding words t and t + 8 of the row) writes the row's 128 terms
+// k_c / max(||k||, eps) -- k_c itself when `raw` -- to out[0..128) in channel order (when `store`).  The whole
+// warp must call (the norm uses the 8-lane butterfly).
+__device__ __forceinline__ void row_terms(const uint4& a, const uint4& b, int t, float inv_eps, bool raw, bool store, float* out) {
+    float2 x[8];
+    unpack_pairs(a, b, x);
+    const float inv = raw ? 1.0f : fminf(approx_rsqrt(pairs_sumsq(x)), inv_eps);
+    if (store) {
+#pragma unroll
+        for (int q = 0; q < 8; q += 2) {
+            // pairs q, q + 1 = four consecutive channels starting at lane_channel(t, 2q)
+            *reinterpret_cast<float4*>(&out[lane_channel(t, 2 * q)]) =
+                make_float4(__fmul_rn(x[q].x, inv), __fmul_rn(x[q].y, inv), __fmul_rn(x[q + 1].x, inv), __fmul_rn(x[q + 1].y, inv));
+        }
+    }
+}
+// terms_sum: staged[j][c] (j < m rows of 128 fp32 terms) summed over j in double; thread (channel c = tid & 127,
+// quarter q = tid >> 7) adds rows q, q + 4, ... in order into acc.  No barrier inside.
+__device__ __forceinline__ void terms_sum(const float* staged, int m, int tid, double& acc) {
+    const int c = tid & (kHeadDim - 1), q = tid >> 7;
+    for (int j = q; j < m; j += 4) acc += static_cast<double>(staged[j * kHeadDim + c]);
+}
+// The four quarters' sums of a channel, in order: returns channel tid's total in threads tid < 128.  part: 4 x 128
+// doubles.  One CTA barrier inside; the caller synchronises before part is reused.
+__device__ __forceinline__ double quarters_sum(double acc, double* part, int tid) {
+    const int c = tid & (kHeadDim - 1), q = tid >> 7;
+    part[q * kHeadDim + c] = acc;
+    __syncthreads();
+    return tid < kHeadDim ? (part[c] + part[kHeadDim + c]) + (part[2 * kHeadDim + c] + part[3 * kHeadDim + c]) : 0.0;
+}
+constexpr int kTermRows = 32;   // rows of terms staged per round (16 KB)
+constexpr int kStashRows = 48;  // evicted cache rows of a slice kept aside as they are (12 KB); at most kGroups
+// Sum of the terms of `count` rows that can be re-read from global memory (row j at row_of(j); the block rows, which
+// nobody writes): phase 1, row group g computes 1/||k|| of rows g, g + 64, ... into inv_sh; phase 2, thread
+// (channel, quarter) re-reads its channel's element of rows q, q + 4, ... and adds the same fp32 products as
+// row_terms forms, in double.  Returns channel tid's sum in threads tid < 128.  All threads call (uniform count);
+// inv_sh: 128 floats, part: 4 x 128 doubles; the caller synchronises before the scratch is reused.
+struct ContiguousRows {   // row j of a run of rows that lie one after the other
+    const uint4* first;
+    __device__ __forceinline__ const uint4* operator()(int j) const { return first + static_cast<size_t>(j) * kRowVec; }
+};
+template <typename RowOf>
+__device__ __forceinline__ double global_rows_terms_sum(RowOf row_of, int count, float inv_eps, bool raw,
+                                                        float* inv_sh, double* part, int tid) {
+    const int g = tid >> 3, t = tid & 7, warp = tid >> 5, c = tid & (kHeadDim - 1), q = tid >> 7;
+    double acc = 0.0;
+    for (int c0 = 0; c0 < count; c0 += kHeadDim) {
+        const int m = min(kHeadDim, count - c0);
+        if (c0 > 0) __syncthreads();   // phase 2 of the previous chunk has read inv_sh
+        for (int j0 = 0; j0 + 4 * warp < m; j0 += kGroups) {   // (warp-uniform bound: pairs_sumsq shuffles)
+            const int j = j0 + g;
+            uint4 a = make_uint4(0, 0, 0, 0), b = a;
+            if (j < m) { const uint4* row = row_of(c0 + j); a = row[t]; b = row[t + 8]; }
+            float2 x[8];
+            unpack_pairs(a, b, x);
+            const float ss = pairs_sumsq(x);
+            if (j < m && t == 0) inv_sh[j] = raw ? 1.0f : fminf(approx_rsqrt(ss), inv_eps);
+        }
+        __syncthreads();
+        for (int jb = q; jb < m; jb += 32) {   // eight rows' elements requested before the first is used
+            uint32_t h[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int j = jb + 4 * i;
+                h[i] = j < m ? __ldg(reinterpret_cast<const uint16_t*>(row_of(c0 + j)) + c) : 0u;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int j = jb + 4 * i;
+                if (j < m) acc += static_cast<double>(__fmul_rn(__uint_as_float(h[i] << 16), inv_sh[j]));
+            }
+        }
+    }
+    return quarters_sum(acc, part, tid);
+}
+
+// Evicted tokens before each word of the bitmap: wlocal[w] = number of set bits in words [0, w).  All threads
+// call; uses sel.warp_gt, sel.hist[32..48) and misc[5], misc[6]; ends with a CTA barrier.
+__device__ __forceinline__ void bitmap_prefix(const uint32_t* bitmap, int nwords, int* wlocal, SelectSmem& sel, int* misc) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int* wbase = sel.hist + 2 * kFusedWarps;
+    for (int w0 = 0; w0 < nwords; w0 += kFusedThreads) {
+        const int wi = w0 + tid;
+        const int pc = wi < nwords ? __popc(bitmap[wi]) : 0;
+        int incl = pc;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) sel.warp_gt[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            const int t2 = lane < kFusedWarps ? sel.warp_gt[lane] : 0;
+            int incl2 = t2;
+#pragma unroll
+            for (int o = 1; o < 16; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl2, o); if (lane >= o) incl2 += v; }
+            if (lane < kFusedWarps) wbase[lane] = incl2 - t2 + (w0 > 0 ? misc[5] : 0);
+            if (lane == kFusedWarps - 1) misc[6] = incl2 + (w0 > 0 ? misc[5] : 0);
+        }
+        __syncthreads();
+        if (wi < nwords) wlocal[wi] = wbase[warp] + incl - pc;   // evicted tokens before word wi
+        if (tid == 0) misc[5] = misc[6];
+        __syncthreads();
+    }
+}
+
+// ||mu|| from the fp32 anchor in shared memory, computed by every warp in the same order.
+__device__ __forceinline__ float anchor_norm(const float* mu, int lane) {
+    const float4 c4 = reinterpret_cast<const float4*>(mu)[lane];
+    float v = fmaf(c4.w, c4.w, fmaf(c4.z, c4.z, fmaf(c4.y, c4.y, c4.x * c4.x)));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return sqrtf(v);
+}
+// Steps a1 + a2 for one landed tile when the anchor is known beforehand: norm and dot product of its 16 rows in
+// one pass, four rows per row group; the keys go to keys_seg[local row].  The whole warp calls.
+__device__ __forceinline__ void score_tile(const uint4* rows, int tile, int rs, int t, int sub, const float2 (&w)[8], float m,
+                                           float eps, uint32_t* keys_seg) {
+    float vs[4];   // this lane's shares of the tile's four rows of its row group
+    double vd[4];
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int lr = tile * kTileRows + it * 4 + sub;
+        uint4 a = make_uint4(0, 0, 0, 0), b = a;
+        if (lr < rs) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
+        lane_sumsq_dot(a, b, w, vs[it], vd[it]);
+    }
+    const uint32_t key = score4(vs, vd, t, m, eps);
+    const int lr = tile * kTileRows + (t >> 1) * 4 + sub;
+    if (!(t & 1) && lr < rs) keys_seg[lr] = key;   // (both lanes of a pair hold the row's key)
+}
+
 // kRegRows = rows per row group that live in registers (the host picks the smallest instance that
 // holds a slice together with the shared-memory rows).
 //
-// kOnePass: the anchor is known before the keys are read.  The library keeps, per unit, the sum of
-// k/||k|| over the rows in the cache (App. B.1, expr. 1, split over time): a step's sum over its n rows
-// is that running sum plus the sum over the B block rows, so only the block has to be normalised
-// before scoring, norm and dot product of a row are taken in one pass while the tiles land, and the
-// first cluster barrier, the anchor exchange and the second pass over the rows disappear.  Every step
-// (either kind) subtracts the evicted rows' k/||k|| again: each CTA leaves the change it saw in
-// anchor_delta, and the next step folds the deltas into the running sum in double precision, in a
-// fixed order.  kOnePass = false recomputes the anchor from all n rows (first evicting step, after
-// set_len / reset / appends, and periodically to shed rounding drift).
+// kOnePass: the anchor is known before the keys are scored.  The library keeps, per unit, the sum of the terms
+// k/||k|| over the rows in the cache (App. B.1, expr. 1, split over time): a step's sum over its n rows is that
+// running sum plus the sum over the B block rows, so only the block has to be normalised before scoring, norm
+// and dot product of a row are taken in one pass, and the first cluster barrier, the anchor exchange and the
+// second pass over the rows disappear.  The anchor of the cluster's NEXT unit is formed while this unit's V rows
+// are on their way in, and the next unit's K tiles are scored by the warp that owns them as soon as they have
+// landed behind the V rows going out: the scoring runs under the copies instead of after them.  Every step
+// (either kind) subtracts the evicted rows' terms again: each CTA leaves the change it saw in anchor_delta, and
+// the next step folds the deltas into the running sum, in double precision and in a fixed order.
+// kOnePass = false recomputes the anchor from all n rows (first evicting step, after set_len / reset / appends,
+// and periodically).
 template <int kRegRows, bool kOnePass>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const FusedParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -434,16 +754,30 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     uint4* rows = reinterpret_cast<uint4*>(smem + L.rows);
     uint32_t* keys = reinterpret_cast<uint32_t*>(smem + L.keys);
     int* hist = reinterpret_cast<int*>(smem + L.work);
-    float* red = reinterpret_cast<float*>(smem + L.work);
     int* dst_of = reinterpret_cast<int*>(smem + L.work);
-    float* partials = reinterpret_cast<float*>(smem + L.xchg);          // [C][128], filled by the peers
+    double* partials = reinterpret_cast<double*>(smem + L.xchg + 2 * kCandCap * 4);   // [C][128], filled by the peers: the anchor
+                                                                                    // partials of a two-pass step, the shares of the
+                                                                                    // next unit's block sum in a one-pass step
     uint32_t* cand_key = reinterpret_cast<uint32_t*>(smem + L.xchg);
     int* cand_idx = reinterpret_cast<int*>(smem + L.xchg) + kCandCap;
     SelectSmem& sel = *reinterpret_cast<SelectSmem*>(smem + L.sel);
-    float* mu_sh = reinterpret_cast<float*>(smem + L.mu);
-    int* misc = reinterpret_cast<int*>(smem + L.misc);   // 0 ncand, 1 first_evicted, 2 need_eq, 3 threshold key
+    float* mu_buf = reinterpret_cast<float*>(smem + L.mu);   // two anchors: this unit's and the next unit's
+    int* misc = reinterpret_cast<int*>(smem + L.misc);   // 0 ncand, 1 first_evicted, 2 need_eq, 3 threshold key, 5/6 prefix carry
     const uint32_t rows_sa = smem_addr(rows), mbar_sa = smem_addr(smem + L.mbar);
     const uint32_t keys_sa = smem_addr(keys), partials_sa = smem_addr(partials);
+    // scratch that the dead key table lends between the selection and the third cluster barrier (no peer writes the
+    // table in that window).  Either the evicted cache rows of the slice are stashed as they are (the K stores put
+    // them there) and turned into terms while the V rows arrive, or -- more of them than the stash holds -- their
+    // terms are staged in rounds before the K stores.
+    uint4* stash = reinterpret_cast<uint4*>(keys);                                     // [kStashRows][16]
+    float* inv_st = reinterpret_cast<float*>(stash + kStashRows * kRowVec);            // [kStashRows]
+    float* inv_ev = inv_st + kStashRows;                                               // [128] evicted block rows of this CTA's range
+    float* inv_nx = inv_ev + kHeadDim;                                                 // [128] the next unit's block rows of that range
+    double* part_g = reinterpret_cast<double*>(inv_nx + kHeadDim);                     // [4][128]
+    double* part_n = part_g + 4 * kHeadDim;                                            // [4][128]
+    float* staged = reinterpret_cast<float*>(keys);                                    // [kTermRows][128]  (rounds only)
+    double* part_gone = reinterpret_cast<double*>(staged + kTermRows * kHeadDim);      // [4][128]
+    int* ev_round = reinterpret_cast<int*>(part_gone + 4 * kHeadDim);                  // [kTermRows]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = tid >> 3, t = tid & 7, sub = lane >> 3;
     const int crank = static_cast<int>(cluster_ctarank());
@@ -451,14 +785,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     const int len = p.len, B = p.B, N = p.N, n = len + B, E = n - N;   // E tokens are evicted
     const float inv_eps = 1.0f / p.eps;
     const bool raw = p.raw_anchor != 0;
-    // fast select: evicted-token bitmap, its per-word prefix and the threshold bin's keys share `xchg`
     const int nwords = (n + 31) >> 5;
-    uint32_t* bitmap = reinterpret_cast<uint32_t*>(smem + L.xchg);
-    int* wlocal = reinterpret_cast<int*>(smem + L.xchg) + nwords;
-    uint32_t* fcand_key = reinterpret_cast<uint32_t*>(smem + L.xchg) + 2 * nwords;
-    int* fcand_idx = reinterpret_cast<int*>(smem + L.xchg) + 2 * nwords + kFastCandCap;
-    const bool fast_ok = n <= kFastKeys * kFusedThreads &&
-                         2 * nwords + 2 * kFastCandCap <= max(C * kHeadDim, 2 * kCandCap);   // uniform over the grid
+    uint32_t* bitmap = reinterpret_cast<uint32_t*>(smem + L.bitmap);
+    int* wlocal = reinterpret_cast<int*>(smem + L.bitmap) + ((p.nkeys + 31) >> 5);
+    const bool fast_ok = n <= kFastKeys * kFusedThreads;   // uniform over the grid
     Slice sl;
     sl.seg_a = min(n, crank * p.rows_per_cta);
     sl.seg = min(n, sl.seg_a + p.rows_per_cta) - sl.seg_a;
@@ -487,9 +817,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         for (int spin = 0; spin < (1 << 16) && global_timer_ns() - t0 < wait_ns; ++spin) __nanosleep(100);
     }
 
+    KD_STAMP_DECL
     constexpr int kRegSlots = kRegRows > 0 ? kRegRows : 1;   // no zero-sized arrays in device code
     uint4 ra[kRegSlots], rb[kRegSlots];   // register-resident rows: local row rs + 64k + g
-    float rn[kRegSlots];
     // K of the cluster's first unit: tiles by the copy engine, the rest by plain loads
     if (cluster_id < p.U) {
         if (lane < kTilesPerWarp && warp + kFusedWarps * lane < ntiles)
@@ -505,173 +835,141 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         }
     }
 
+    // One-pass steps.  The B block rows of a unit are normalised once per cluster: CTA r takes block rows
+    // [b_lo, b_hi), pushes its share of their sum of terms into every peer's table (DSMEM), and after a cluster
+    // barrier every CTA adds the C shares in rank order to the folded running sum: the same anchor bits everywhere.
+    const int b_per = (B + C - 1) / C;
+    const int b_lo = min(B, crank * b_per), b_hi = min(B, b_lo + b_per), nb = b_hi - b_lo;
+    double my_share = 0.0;       // tid < 128: channel tid of this CTA's share of this unit's block sum
+    double folded = 0.0;         // tid < 128: channel tid of this unit's folded running sum (cached rows)
+    bool tiles_scored = false;   // this unit's tiles were scored behind the previous unit's V rows
+    int cur = 0;                 // which of the two anchor buffers holds this unit's anchor
+    auto fold_running_sum = [&](int uu) -> double {   // threads tid < 128
+        double a = p.anchor_in[static_cast<size_t>(uu) * kHeadDim + tid];
+        double dl[kMaxCluster];
+#pragma unroll
+        for (int c = 0; c < kMaxCluster; ++c)
+            dl[c] = c < C ? p.anchor_delta[(static_cast<size_t>(uu) * C + c) * kHeadDim + tid] : 0.0;
+#pragma unroll
+        for (int c = 0; c < kMaxCluster; ++c) a += dl[c];   // rank order; absent ranks add 0
+        if (crank == 0) p.anchor_out[static_cast<size_t>(uu) * kHeadDim + tid] = a;   // the cached rows' sum, folded
+        return a;
+    };
+    auto push_share = [&](double v) {   // threads tid < 128: this CTA's row of every peer's table
+        const uint32_t slot = partials_sa + 8 * (crank * kHeadDim + tid);
+        for (int c = 0; c < C; ++c) st_cluster_f64(map_to_cta(slot, c), v);
+    };
+    auto anchor_from_shares = [&](double a, float* mu_out) {   // threads tid < 128, after the cluster barrier
+        double bs = 0.0;
+        for (int c = 0; c < C; ++c) bs += partials[c * kHeadDim + tid];
+        mu_out[tid] = static_cast<float>((a + bs) / static_cast<double>(n));
+    };
+    if (kOnePass && cluster_id < p.U) {   // the first unit's anchor (the work area is free before the first unit)
+        if (tid < kHeadDim) folded = fold_running_sum(cluster_id);
+        const ContiguousRows blk{p.new_k + (static_cast<size_t>(cluster_id) * B + b_lo) * kRowVec};
+        my_share = global_rows_terms_sum(blk, nb, inv_eps, raw, reinterpret_cast<float*>(smem + L.work) + 8 * kHeadDim,
+                                         reinterpret_cast<double*>(smem + L.work), tid);
+        if (tid < kHeadDim) push_share(my_share);
+        cluster_sync_all();
+        if (tid < kHeadDim) anchor_from_shares(folded, mu_buf);
+        __syncthreads();
+    }
+
+    KD_STAMP(0);
     for (int u = cluster_id; u < p.U; u += nclusters) {
         const int un = u + nclusters;   // the unit this cluster serves next
-        float block_sum = 0.f;   // tid < 128: channel tid of the block rows' sum of k/||k||
+        float* mu_sh = mu_buf + cur * kHeadDim;
         if constexpr (kOnePass) {
-        // ------------------------------------------------------------ anchor from the running sum + the block rows
-        {
-            // the running sum and its pending deltas, requested first: they arrive under the block's arithmetic
-            double run = 0.0;
-            float dl[kMaxCluster];
-            if (tid < kHeadDim) {
-                run = p.anchor_in[static_cast<size_t>(u) * kHeadDim + tid];
-#pragma unroll
-                for (int c = 0; c < kMaxCluster; ++c)
-                    dl[c] = c < C ? p.anchor_delta[(static_cast<size_t>(u) * C + c) * kHeadDim + tid] : 0.f;
-            }
-            float2 acc[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) acc[q] = make_float2(0.f, 0.f);
-            for (int b0 = 0; b0 < B; b0 += kGroups) {   // every CTA normalises the whole block: no exchange needed
-                const int br = b0 + g;                   // (same trip count in every lane: row_a1 shuffles)
-                uint4 a = make_uint4(0, 0, 0, 0), b = a;
-                if (br < B) {
-                    const uint4* row = p.new_k + (static_cast<size_t>(u) * B + br) * kRowVec;
-                    a = row[t]; b = row[t + 8];
-                }
-                row_a1(a, b, br < B, inv_eps, acc, raw);
-            }
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                float2 v = acc[q];
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
-                acc[q] = v;
-            }
-            if (lane < 8) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    *reinterpret_cast<float2*>(&red[warp * kHeadDim + lane_channel(t, 2 * q)]) = acc[q];
-            }
-            __syncthreads();
-            if (tid < kHeadDim) {
-#pragma unroll
-                for (int w = 0; w < kFusedWarps; ++w) block_sum += red[w * kHeadDim + tid];
-                double a = run;
-#pragma unroll
-                for (int c = 0; c < kMaxCluster; ++c) a += static_cast<double>(dl[c]);   // rank order; absent ranks add 0
-                if (crank == 0) p.anchor_out[static_cast<size_t>(u) * kHeadDim + tid] = a;   // the cached rows' sum, folded
-                mu_sh[tid] = static_cast<float>((a + static_cast<double>(block_sum)) / static_cast<double>(n));
-            }
-            __syncthreads();
-        }
-        // ------------------------------------------------------------ a1 + a2 in one pass: keys of this slice
-        {
+            // ------------------------------------------------------------ a1 + a2 in one pass: keys of this slice
             float2 w[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) w[q] = *reinterpret_cast<const float2*>(&mu_sh[lane_channel(t, 2 * q)]);
-            float m;   // ||mu||, computed by every warp in the same order
-            {
-                const float4 c4 = reinterpret_cast<const float4*>(mu_sh)[lane];
-                float v = fmaf(c4.w, c4.w, fmaf(c4.z, c4.z, fmaf(c4.y, c4.y, c4.x * c4.x)));
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                m = sqrtf(v);
+            load_anchor(mu_sh, t, w);
+            const float m = anchor_norm(mu_sh, lane);
+            if (!tiles_scored) {
+#pragma unroll 1
+                for (int s = 0; s < kTilesPerWarp; ++s) {
+                    const int tile = warp + kFusedWarps * s;
+                    if (tile >= ntiles) break;
+                    mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
+                    parity ^= 1u << s;
+                    score_tile(rows, tile, rs, t, sub, w, m, p.eps, keys + seg_a);
+                }
             }
+#pragma unroll
+            for (int k0 = 0; k0 < kRegRows; k0 += 4) {   // register rows, four at a time
+                float vs[4];
+                double vd[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (k0 + i < kRegRows) lane_sumsq_dot(ra[k0 + i], rb[k0 + i], w, vs[i], vd[i]);
+                    else { vs[i] = 0.f; vd[i] = 0.0; }
+                }
+                const uint32_t key = score4(vs, vd, t, m, p.eps);
+                const int lr = rs + (k0 + (t >> 1)) * kGroups + g;
+                if (!(t & 1) && k0 + (t >> 1) < kRegRows && lr < seg) keys[seg_a + lr] = key;
+            }
+        } else {
+            // ------------------------------------------------------------ a1: norms and anchor partial
+            float rn[kRegSlots];
+            double wide[16];   // this thread's sums, carried in double above the four rows of a tile
+#pragma unroll
+            for (int j = 0; j < 16; ++j) wide[j] = 0.0;
 #pragma unroll 1
             for (int s = 0; s < kTilesPerWarp; ++s) {
                 const int tile = warp + kFusedWarps * s;
                 if (tile >= ntiles) break;
                 mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
                 parity ^= 1u << s;
-                float v[8];   // this lane's shares of the tile's four rows of its row group
+                float2 acc[8];
 #pragma unroll
-                for (int it = 0; it < 4; ++it) {
-                    const int lr = tile * kTileRows + it * 4 + sub;
-                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
-                    if (lr < rs) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
-                    lane_sumsq_dot(a, b, w, v[2 * it], v[2 * it + 1]);
-                }
-                const uint32_t key = score4(v, t, m, p.eps);
-                const int lr = tile * kTileRows + (t >> 1) * 4 + sub;
-                if (!(t & 1) && lr < rs) keys[seg_a + lr] = key;
-            }
-#pragma unroll
-            for (int k0 = 0; k0 < kRegRows; k0 += 4) {   // register rows, four at a time
-                float v[8];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    if (k0 + i < kRegRows) lane_sumsq_dot(ra[k0 + i], rb[k0 + i], w, v[2 * i], v[2 * i + 1]);
-                    else { v[2 * i] = 0.f; v[2 * i + 1] = 0.f; }
-                }
-                const uint32_t key = score4(v, t, m, p.eps);
-                const int lr = rs + (k0 + (t >> 1)) * kGroups + g;
-                if (!(t & 1) && k0 + (t >> 1) < kRegRows && lr < seg) keys[seg_a + lr] = key;
-            }
-        }
-        } else {
-        // ------------------------------------------------------------ a1: norms and anchor partial
-        float2 acc[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) acc[q] = make_float2(0.f, 0.f);
+                for (int q = 0; q < 8; ++q) acc[q] = make_float2(0.f, 0.f);
 #pragma unroll 1
-        for (int s = 0; s < kTilesPerWarp; ++s) {
-            const int tile = warp + kFusedWarps * s;
-            if (tile >= ntiles) break;
-            mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
-            parity ^= 1u << s;
-#pragma unroll 1
-            for (int half = 0; half < 2; ++half) {
-                uint4 a[2], b[2];
+                for (int half = 0; half < 2; ++half) {
+                    uint4 a[2], b[2];
 #pragma unroll
-                for (int it = 0; it < 2; ++it) {
-                    const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
-                    a[it] = make_uint4(0, 0, 0, 0); b[it] = a[it];
-                    if (lr < rs) { a[it] = rows[lr * kRowVec + t]; b[it] = rows[lr * kRowVec + t + 8]; }
+                    for (int it = 0; it < 2; ++it) {
+                        const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
+                        a[it] = make_uint4(0, 0, 0, 0); b[it] = a[it];
+                        if (lr < rs) { a[it] = rows[lr * kRowVec + t]; b[it] = rows[lr * kRowVec + t + 8]; }
+                    }
+#pragma unroll
+                    for (int it = 0; it < 2; ++it) {
+                        const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
+                        const float r = row_a1(a[it], b[it], lr < rs, inv_eps, acc, raw);
+                        if (lr < rs && t == 0) keys[seg_a + lr] = __float_as_uint(r);   // parked in the row's key slot until a2
+                    }
                 }
 #pragma unroll
-                for (int it = 0; it < 2; ++it) {
-                    const int lr = tile * kTileRows + (2 * half + it) * 4 + sub;
-                    const float r = row_a1(a[it], b[it], lr < rs, inv_eps, acc, raw);
-                    if (lr < rs && t == 0) keys[seg_a + lr] = __float_as_uint(r);   // parked in the row's key slot until a2
-                }
+                for (int q = 0; q < 8; ++q) { wide[2 * q] += static_cast<double>(acc[q].x); wide[2 * q + 1] += static_cast<double>(acc[q].y); }
             }
-        }
-#pragma unroll
-        for (int k = 0; k < kRegRows; ++k) rn[k] = row_a1(ra[k], rb[k], rs + k * kGroups + g < seg, inv_eps, acc, raw);
-        // CTA reduction: 4 groups of a warp by shuffle, 16 warps through shared memory, fixed order
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            float2 v = acc[q];
-            v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
-            v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
-            acc[q] = v;
-        }
-        if (lane < 8) {
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                *reinterpret_cast<float2*>(&red[warp * kHeadDim + lane_channel(t, 2 * q)]) = acc[q];
-        }
-        __syncthreads();
-        if (tid < kHeadDim) {
-            float s = 0.f;
-#pragma unroll
-            for (int w = 0; w < kFusedWarps; ++w) s += red[w * kHeadDim + tid];
-            const uint32_t slot = partials_sa + 4 * (crank * kHeadDim + tid);
-            for (int c = 0; c < C; ++c) st_cluster_f32(map_to_cta(slot, c), s);   // this CTA's row of every peer's table
-        }
-        cluster_sync_all();   // (1) all partials delivered; every K row of the unit is on chip
-        if (tid < kHeadDim) {
-            float s = 0.f;
-            for (int c = 0; c < C; ++c) s += partials[c * kHeadDim + tid];   // rank order: same bits in every CTA
-            mu_sh[tid] = s / static_cast<float>(n);
-            if (crank == 0) p.anchor_out[static_cast<size_t>(u) * kHeadDim + tid] = static_cast<double>(s);   // sum over all n rows
-        }
-        __syncthreads();
-        // ------------------------------------------------------------ a2: keys of this slice into the table
-        {
-            float2 w[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) w[q] = *reinterpret_cast<const float2*>(&mu_sh[lane_channel(t, 2 * q)]);
-            float m;   // ||mu||, computed by every warp in the same order
             {
-                const float4 c4 = reinterpret_cast<const float4*>(mu_sh)[lane];
-                float v = fmaf(c4.w, c4.w, fmaf(c4.z, c4.z, fmaf(c4.y, c4.y, c4.x * c4.x)));
+                float2 acc[8];
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                m = sqrtf(v);
+                for (int q = 0; q < 8; ++q) acc[q] = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int k = 0; k < kRegRows; ++k) rn[k] = row_a1(ra[k], rb[k], rs + k * kGroups + g < seg, inv_eps, acc, raw);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) { wide[2 * q] += static_cast<double>(acc[q].x); wide[2 * q + 1] += static_cast<double>(acc[q].y); }
             }
+            // CTA reduction in double (the key table holds the parked norms, so the 8 KB work area serves, in two rounds)
+            {
+                const double s = cta_channel_sum<1>(wide, reinterpret_cast<double*>(smem + L.work), tid);
+                if (tid < kHeadDim) {
+                    const uint32_t slot = partials_sa + 8 * (crank * kHeadDim + tid);
+                    for (int c = 0; c < C; ++c) st_cluster_f64(map_to_cta(slot, c), s);   // this CTA's row of every peer's table
+                }
+            }
+            cluster_sync_all();   // (1) all partials delivered; every K row of the unit is on chip
+            if (tid < kHeadDim) {
+                double s = 0.0;
+                for (int c = 0; c < C; ++c) s += partials[c * kHeadDim + tid];   // rank order: same bits in every CTA
+                mu_sh[tid] = static_cast<float>(s / static_cast<double>(n));
+                if (crank == 0) p.anchor_out[static_cast<size_t>(u) * kHeadDim + tid] = s;   // sum over all n rows
+            }
+            __syncthreads();
+            // ------------------------------------------------------------ a2: keys of this slice into the table
+            float2 w[8];
+            load_anchor(mu_sh, t, w);
+            const float m = anchor_norm(mu_sh, lane);
 #pragma unroll 1
             for (int s = 0; s < kTilesPerWarp; ++s) {
                 const int tile = warp + kFusedWarps * s;
@@ -700,8 +998,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 const int lr = rs + k * kGroups + g;
                 if (lr < seg && t == 0) keys[seg_a + lr] = key;
             }
-        }
         }   // kOnePass
+        KD_STAMP(1);
         __syncthreads();
         {
             // this slice's keys -> every peer's table (128-bit DSMEM stores)
@@ -716,13 +1014,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         {
             float* sc = p.scores + static_cast<size_t>(u) * p.nmax + seg_a;   // fp32 scores to global scratch, coalesced
             for (int lr = tid; lr < seg; lr += kFusedThreads) sc[lr] = key_score(keys[seg_a + lr]);
-            if (fast_ok) {
-                for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;          // `red` is dead
-                for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;   // the partials are dead
-                if (tid == 0) { misc[0] = 0; misc[1] = n; }
-            }
+            for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;
+            for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;
+            if (tid == 0) { misc[0] = 0; misc[1] = n; }
         }
         cluster_wait();       // (2) the key table of every CTA holds all n keys
+        KD_STAMP(2);
         if (p.window > 0) {
             // sliding window (Sec. 3.2): the last `window` tokens get the largest possible key, so they are
             // never among the E smallest; the scores in global scratch stay what they are
@@ -731,126 +1028,25 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             __syncthreads();
         }
         // ------------------------------------------------------------ a3 + plan: who is evicted, where every kept row goes
-        bool planned = false;
-        if (fast_ok) {
-            // Only E keys go, so the work is at the low end.  Thread t keeps the keys of tokens t, t+512, ...
-            // in registers; the 2048 bins are spread over the low end of the unit's own key range (from the
-            // smallest key to a bound on the E-th smallest; monotone in the key, which is all selection needs); the
-            // tokens under the threshold bin go straight into a bitmap, the bin's own few keys are ranked
-            // exactly, and prefix counts over the bitmap give every kept row of the slice its destination.
-            uint32_t* wmin = reinterpret_cast<uint32_t*>(sel.hist);          // (sel.hist is radix-select scratch)
-            uint32_t* wmax = reinterpret_cast<uint32_t*>(sel.hist) + kFusedWarps;
-            int* wbase = sel.hist + 2 * kFusedWarps;
-            const int cnt = (n - tid + kFusedThreads - 1) / kFusedThreads;
-            uint32_t kk[kFastKeys];
-#pragma unroll
-            for (int j = 0; j < kFastKeys; ++j) kk[j] = j < cnt ? keys[tid + j * kFusedThreads] : 0xffffffffu;
-            {
-                uint32_t lo = 0xffffffffu, hi = 0u;
-#pragma unroll
-                for (int j = 0; j < kFastKeys; ++j) { lo = min(lo, kk[j]); if (j < cnt) hi = max(hi, kk[j]); }
-                // The E-th smallest key is at most the largest of any E distinct keys.  When at least E
-                // threads hold keys, the thread minima are such keys, so the largest thread minimum bounds
-                // it; otherwise the largest key does.  Keys above the bound share the top bin.
-                const uint32_t cut = (n >= kFusedThreads && E <= kFusedThreads) ? lo : hi;
-                const uint32_t wlo = __reduce_min_sync(0xffffffffu, lo);
-                const uint32_t wcut = __reduce_max_sync(0xffffffffu, cnt > 0 ? cut : 0u);
-                if (lane == 0) { wmin[warp] = wlo; wmax[warp] = wcut; }
+        {
+            // the evicted tokens' bits: selection at the low end of the table, or (crowded threshold bin, large
+            // unit) the full-table route; then prefix counts over the bitmap give every kept row of the slice
+            // its destination
+            const bool planned = fast_ok && low_end_select(keys, n, E, hist, bitmap, cand_key, cand_idx, sel, misc);
+            if (!planned) {
+                for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;   // (the attempt may have marked some)
+                __syncthreads();
+                full_select_plan(keys, n, N, 0, 0, hist, cand_key, cand_idx, nullptr, sel, misc, bitmap);
+            }
+            bitmap_prefix(bitmap, nwords, wlocal, sel, misc);
+            for (int lr = tid; lr < seg; lr += kFusedThreads) {
+                const int i = seg_a + lr, w = i >> 5;
+                const uint32_t wd = bitmap[w], bit = 1u << (i & 31);
+                dst_of[lr] = (wd & bit) ? -1 : i - (wlocal[w] + __popc(wd & (bit - 1)));
             }
             __syncthreads();
-            uint32_t kmin, kcut, shift;
-            {
-                const uint32_t lo = lane < kFusedWarps ? wmin[lane] : 0xffffffffu, hi = lane < kFusedWarps ? wmax[lane] : 0u;
-                kmin = __reduce_min_sync(0xffffffffu, lo);
-                kcut = __reduce_max_sync(0xffffffffu, hi);
-                const int bits = 32 - __clz(kcut - kmin);   // significant bits of the range [kmin, kcut]
-                shift = bits > 11 ? bits - 11 : 0;          // (key - kmin) >> shift < 2048 inside the range
-            }
-            // bin of a key: linear in the key over [kmin, kcut] (bins 0..2046), 2047 above; monotone
-            auto bin_of = [kmin, kcut, shift](uint32_t k) { return k <= kcut ? min((k - kmin) >> shift, 2046u) : 2047u; };
-#pragma unroll
-            for (int j = 0; j < kFastKeys; ++j) {
-                // (the top bin holds every key above the bound: the crossing is never there, so it is not counted)
-                const uint32_t b = bin_of(kk[j]);
-                if (j < cnt && b != 2047u) atomicAdd(&hist[b], 1);
-            }
-            __syncthreads();
-            const int packed = find_crossing(hist, E, lane, warp, sel.warp_eq);
-            const uint32_t bstar = static_cast<uint32_t>(packed >> 16);
-            const int need = E - (packed & 0xffff);   // this many keys of the threshold bin go
-            unsigned m_below = 0, m_in = 0;           // bit j: this thread's j-th key is below / inside the bin
-#pragma unroll
-            for (int j = 0; j < kFastKeys; ++j) {
-                const uint32_t b = bin_of(kk[j]);
-                m_below |= (j < cnt && b < bstar) ? 1u << j : 0u;
-                m_in |= (j < cnt && b == bstar) ? 1u << j : 0u;
-            }
-            {
-                int first = n;
-                if (packed >= 0 && (m_below | m_in)) {
-                    for (unsigned m = m_below; m; m &= m - 1) {
-                        const int i = tid + (__ffs(m) - 1) * kFusedThreads;
-                        atomicOr(&bitmap[i >> 5], 1u << (i & 31));
-                        first = min(first, i);
-                    }
-                    for (unsigned m = m_in; m; m &= m - 1) {
-                        const int i = tid + (__ffs(m) - 1) * kFusedThreads;
-                        const int slot = atomicAdd(&misc[0], 1);
-                        if (slot < kFastCandCap) { fcand_key[slot] = keys[i]; fcand_idx[slot] = i; }
-                    }
-                }
-                first = __reduce_min_sync(0xffffffffu, first);   // one shared-memory atomic per warp, not per thread
-                if (lane == 0 && first < n) atomicMin(&misc[1], first);
-            }
-            __syncthreads();
-            const int ncand = misc[0];
-            if (packed >= 0 && ncand <= kFastCandCap) {   // uniform: every thread sees the same values
-                // Eviction order is the reverse of the keep order: key ascending, index descending.
-                int wfirst = n;
-                for (int c = warp; c < ncand; c += kFusedWarps) {
-                    const uint32_t mk = fcand_key[c];
-                    const int mi = fcand_idx[c];
-                    int rank = 0;
-                    for (int q = lane; q < ncand; q += 32) {
-                        const uint32_t ok = fcand_key[q];
-                        rank += (ok < mk) || (ok == mk && fcand_idx[q] > mi);
-                    }
-                    rank = __reduce_add_sync(0xffffffffu, rank);
-                    if (lane == 0 && rank < need) { atomicOr(&bitmap[mi >> 5], 1u << (mi & 31)); wfirst = min(wfirst, mi); }
-                }
-                if (lane == 0 && wfirst < n) atomicMin(&misc[1], wfirst);
-                __syncthreads();
-                {
-                    // evicted tokens before each word of the bitmap: one word per thread (nwords <= 512)
-                    const int pc = tid < nwords ? __popc(bitmap[tid]) : 0;
-                    int incl = pc;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                        if (lane >= o) incl += v;
-                    }
-                    if (tid < nwords) wlocal[tid] = incl - pc;
-                    if (lane == 31) sel.warp_gt[warp] = incl;
-                }
-                __syncthreads();
-                if (warp == 0) {
-                    const int t2 = lane < kFusedWarps ? sel.warp_gt[lane] : 0;
-                    int incl = t2;
-#pragma unroll
-                    for (int o = 1; o < 16; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += v; }
-                    if (lane < kFusedWarps) wbase[lane] = incl - t2;
-                }
-                __syncthreads();
-                for (int lr = tid; lr < seg; lr += kFusedThreads) {
-                    const int i = seg_a + lr, w = i >> 5;
-                    const uint32_t wd = bitmap[w], bit = 1u << (i & 31);
-                    dst_of[lr] = (wd & bit) ? -1 : i - (wbase[w >> 5] + wlocal[w] + __popc(wd & (bit - 1)));
-                }
-                __syncthreads();
-                planned = true;
-            }
         }
-        if (!planned) full_select_plan(keys, n, N, seg_a, seg_b, hist, cand_key, cand_idx, dst_of, sel, misc);
+        KD_STAMP(3);
         const int first_evicted = misc[1];
         const int first_moved = min(first_evicted, len);   // block rows always move into the cache
         const int skip_local = first_moved - seg_a;        // local rows below this keep their place
@@ -865,25 +1061,70 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 if (p.kept_mirror) p.kept_mirror[static_cast<size_t>(u) * N + d] = seg_a + lr;
             }
         }
+        KD_STAMP(4);
+        // ------------------------------------------------------------ the evicted rows leave the running anchor sum
+        // This CTA's delta to the running sum: its share of the block that came in (one-pass steps) minus the terms
+        // of (a) the evicted cache rows of its slice, which only exist on chip once the K stores have run, and (b)
+        // the evicted block rows of its range of the block, which stay readable in global memory.
+        auto evicted_before = [&](int i) { const int w = i >> 5; return wlocal[w] + __popc(bitmap[w] & ((1u << (i & 31)) - 1u)); };
+        const int c_lo = min(seg_a, len), c_hi = min(seg_b, len);             // the slice's cache rows
+        const int eb_lo = evicted_before(c_lo);                               // (len < n: the index is inside the bitmap)
+        const int n_gone_cache = evicted_before(c_hi) - eb_lo;
+        const bool use_stash = n_gone_cache <= kStashRows;
+        double gone_rounds = 0.0;   // tid < 128 after the rounds
+        if (!use_stash) {
+            // Rounds before the K stores: evicted cache row number j of the slice (ascending) is staged as 128
+            // terms in row j of a round of kTermRows rows.
+            double acc = 0.0;
+            const int w_first = c_lo >> 5;
+            for (int r0 = 0; r0 < n_gone_cache; r0 += kTermRows) {
+                const int cnt = min(kTermRows, n_gone_cache - r0);
+                if (r0 > 0) __syncthreads();   // the previous round's terms and list have been read
+                // which staged row is which local row: one thread per bitmap word (-1: the row lives in registers)
+                if (w_first + tid < nwords && ((w_first + tid) << 5) < c_hi) {
+                    const int w = w_first + tid;
+                    int j = wlocal[w] - eb_lo - r0;
+                    for (uint32_t wd = bitmap[w]; wd; wd &= wd - 1, ++j) {
+                        const int i = 32 * w + __ffs(wd) - 1;
+                        if (i >= c_lo && i < c_hi && j >= 0 && j < kTermRows) ev_round[j] = i - seg_a < rs ? i - seg_a : -1;
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < kRegRows; ++k) {   // register-resident rows: their own row group
+                    const int lr = rs + k * kGroups + g;
+                    const int j = (lr < seg && seg_a + lr < len && dst_of[lr] < 0) ? evicted_before(seg_a + lr) - eb_lo - r0 : -1;
+                    row_terms(ra[k], rb[k], t, inv_eps, raw, j >= 0 && j < kTermRows, staged + max(j, 0) * kHeadDim);
+                }
+                __syncthreads();
+                if (g < kTermRows) {   // (warps 0..7, warp-uniform: row_terms shuffles) row group g takes staged row g
+                    const int lr = g < cnt ? ev_round[g] : -1;
+                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
+                    if (lr >= 0) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
+                    row_terms(a, b, t, inv_eps, raw, lr >= 0, staged + g * kHeadDim);
+                }
+                __syncthreads();
+                terms_sum(staged, cnt, tid, acc);
+            }
+            gone_rounds = quarters_sum(acc, part_gone, tid);
+            __syncthreads();   // the scratch is free for what follows
+        }
         // ------------------------------------------------------------ a4: K rows out, V rows in behind them
         {
             uint4* out = p.k_cache + static_cast<size_t>(u) * N * kRowVec;
-            float2 gone[8];   // sum of k/||k|| over this thread's share of the evicted rows (for the running anchor)
-#pragma unroll
-            for (int q = 0; q < 8; ++q) gone[q] = make_float2(0.f, 0.f);
-            if (kOnePass && crank == 0 && un < p.U) {   // the next unit's block rows towards L2: every CTA reads them first thing
-                const char* nb = reinterpret_cast<const char*>(p.new_k + static_cast<size_t>(un) * B * kRowVec);
+            if (kOnePass && crank == 0 && un + nclusters < p.U) {   // the block rows of the unit after next towards L2
+                const char* nb = reinterpret_cast<const char*>(p.new_k + static_cast<size_t>(un + nclusters) * B * kRowVec);
                 for (int o = tid * 128; o < B * kRowBytes; o += kFusedThreads * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(nb + o));
             }
-            // (row_a1 shuffles inside each row group, so the whole warp enters it together: the vote is
-            // warp-wide, the row's own flag only decides whether it contributes)
 #pragma unroll
             for (int k = 0; k < kRegRows; ++k) {
                 const int lr = rs + k * kGroups + g;
                 const bool vis = lr < seg && lr >= skip_local;
-                const int d = vis ? dst_of[lr] : 0;
-                if (vis && d >= 0) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
-                if (__any_sync(0xffffffffu, vis && d < 0)) row_a1(ra[k], rb[k], vis && d < 0, inv_eps, gone, raw);
+                const int d = vis ? dst_of[lr] : -1;
+                if (d >= 0) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
+                if (vis && d < 0 && use_stash && seg_a + lr < len) {   // an evicted cache row: kept aside as it is
+                    uint4* srow = stash + (evicted_before(seg_a + lr) - eb_lo) * kRowVec;
+                    srow[t] = ra[k]; srow[t + 8] = rb[k];
+                }
                 if (vis) {
                     const uint4* row = concat_row(p.v_cache, p.new_v, u, seg_a + lr, len, B, N);
                     ra[k] = row[t]; rb[k] = row[t + 8];
@@ -894,15 +1135,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 const int tile = warp + kFusedWarps * s;
                 if (tile >= ntiles) break;
                 if (min(rs, (tile + 1) * kTileRows) <= skip_local) continue;   // no row of the tile moves
-#pragma unroll 1
+#pragma unroll
                 for (int it = 0; it < 4; ++it) {
                     const int lr = tile * kTileRows + it * 4 + sub;
                     const bool vis = lr < rs && lr >= skip_local;
-                    const int d = vis ? dst_of[lr] : 0;
-                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
-                    if (vis) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
-                    if (vis && d >= 0) { out[d * kRowVec + t] = a; out[d * kRowVec + t + 8] = b; }
-                    if (__any_sync(0xffffffffu, vis && d < 0)) row_a1(a, b, vis && d < 0, inv_eps, gone, raw);
+                    const int d = vis ? dst_of[lr] : -1;
+                    if (d >= 0) { out[d * kRowVec + t] = rows[lr * kRowVec + t]; out[d * kRowVec + t + 8] = rows[lr * kRowVec + t + 8]; }
+                    if (vis && d < 0 && use_stash && seg_a + lr < len) {   // an evicted cache row: kept aside as it is
+                        uint4* srow = stash + (evicted_before(seg_a + lr) - eb_lo) * kRowVec;
+                        srow[t] = rows[lr * kRowVec + t]; srow[t + 8] = rows[lr * kRowVec + t + 8];
+                    }
                 }
                 // The tile's only readers are this warp's lanes and their reads have returned (the stores
                 // above consumed them), so the copy engine may overwrite it: a write after reads needs
@@ -910,29 +1152,87 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 __syncwarp();
                 if (lane == 0) issue_tile(p.v_cache, p.new_v, u, len, B, N, sl, tile, rows_sa, mbar_sa);
             }
-            // what this CTA saw leave (and, on rank 0 of a one-pass step, the block that came in): its delta
-            // to the running sum.  The key table is dead until the next unit: 8 KB of it serve as scratch.
-            float* red2 = reinterpret_cast<float*>(keys);
+        }
+        KD_STAMP(6);
+        // ------------------------------------------------------------ while the V rows arrive: terms of the rows that left,
+        // and this CTA's share of the next unit's block
+        double folded_next = 0.0, share_next = 0.0;
+        {
+            const bool next_share = kOnePass && un < p.U;
+            if (next_share && tid < kHeadDim) folded_next = fold_running_sum(un);   // (its loads arrive under what follows)
+            __syncthreads();   // the stash is complete
+            const int n_st = use_stash ? n_gone_cache : 0;
+            const uint4* blk_u = p.new_k + static_cast<size_t>(u) * B * kRowVec;
+            const uint4* blk_n = p.new_k + static_cast<size_t>(next_share ? un : u) * B * kRowVec;
+            const int c = tid & (kHeadDim - 1), q = tid >> 7;
+            double gone = 0.0, nxt = 0.0;
+            for (int r0 = b_lo; r0 == b_lo || r0 < b_hi; r0 += kHeadDim) {   // 128 block rows of the range at a time (usually all)
+                const int mc = max(0, min(kHeadDim, b_hi - r0));
+                const int st0 = r0 == b_lo ? n_st : 0;                        // the stash goes with the first chunk
+                const int items = st0 + mc + (next_share ? mc : 0);
+                if (r0 > b_lo) __syncthreads();   // the previous chunk's reciprocal norms have been read
+                // phase 1: one row group per row: 1 / ||k||
+                for (int i0 = 0; i0 + 4 * warp < items; i0 += kGroups) {   // (warp-uniform bound: pairs_sumsq shuffles)
+                    int it = i0 + g;
+                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
+                    float* inv_out = nullptr;
+                    if (it < st0) {
+                        a = stash[it * kRowVec + t]; b = stash[it * kRowVec + t + 8];
+                        inv_out = inv_st + it;
+                    } else if ((it -= st0) < mc) {
+                        const int i = len + r0 + it;   // token index of block row r0 + it
+                        if ((bitmap[i >> 5] >> (i & 31)) & 1u) {
+                            const uint4* row = blk_u + static_cast<size_t>(r0 + it) * kRowVec;
+                            a = row[t]; b = row[t + 8];
+                            inv_out = inv_ev + it;
+                        } else if (t == 0) {
+                            inv_ev[it] = 0.f;   // kept: no term
+                        }
+                    } else if ((it -= mc) < mc && next_share) {
+                        const uint4* row = blk_n + static_cast<size_t>(r0 + it) * kRowVec;
+                        a = row[t]; b = row[t + 8];
+                        inv_out = inv_nx + it;
+                    }
+                    float2 x[8];
+                    unpack_pairs(a, b, x);
+                    const float ss = pairs_sumsq(x);
+                    if (inv_out && t == 0) *inv_out = raw ? 1.0f : fminf(approx_rsqrt(ss), inv_eps);
+                }
+                __syncthreads();
+                // phase 2: thread (channel c, quarter q) adds rows q, q + 4, ... of its channel, in order, in double
+                for (int j = q; j < st0; j += 4) {
+                    const uint32_t h = reinterpret_cast<const uint16_t*>(stash + j * kRowVec)[c];
+                    gone += static_cast<double>(__fmul_rn(__uint_as_float(h << 16), inv_st[j]));
+                }
+                for (int jb = q; jb < mc; jb += 32) {   // eight rows' elements requested before the first is used
+                    uint32_t he[8], hn[8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                float2 v = gone[q];
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
-                gone[q] = v;
-            }
-            if (lane < 8) {
+                    for (int i = 0; i < 8; ++i) {
+                        const int j = jb + 4 * i;
+                        he[i] = (j < mc && inv_ev[j] != 0.f) ? __ldg(reinterpret_cast<const uint16_t*>(blk_u + static_cast<size_t>(r0 + j) * kRowVec) + c) : 0u;
+                        hn[i] = (j < mc && next_share) ? __ldg(reinterpret_cast<const uint16_t*>(blk_n + static_cast<size_t>(r0 + j) * kRowVec) + c) : 0u;
+                    }
 #pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    *reinterpret_cast<float2*>(&red2[warp * kHeadDim + lane_channel(t, 2 * q)]) = gone[q];
+                    for (int i = 0; i < 8; ++i) {
+                        const int j = jb + 4 * i;
+                        if (j < mc && inv_ev[j] != 0.f) gone += static_cast<double>(__fmul_rn(__uint_as_float(he[i] << 16), inv_ev[j]));
+                        if (j < mc && next_share) nxt += static_cast<double>(__fmul_rn(__uint_as_float(hn[i] << 16), inv_nx[j]));
+                    }
+                }
             }
+            part_g[q * kHeadDim + c] = gone;
+            part_n[q * kHeadDim + c] = nxt;
             __syncthreads();
             if (tid < kHeadDim) {
-                float e = 0.f;
-#pragma unroll
-                for (int w = 0; w < kFusedWarps; ++w) e += red2[w * kHeadDim + tid];
-                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass && crank == 0 ? block_sum : 0.f) - e;
+                const double gsum = gone_rounds + ((part_g[c] + part_g[kHeadDim + c]) + (part_g[2 * kHeadDim + c] + part_g[3 * kHeadDim + c]));
+                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass ? my_share : 0.0) - gsum;
+                if (next_share) {
+                    share_next = (part_n[c] + part_n[kHeadDim + c]) + (part_n[2 * kHeadDim + c] + part_n[3 * kHeadDim + c]);
+                    push_share(share_next);   // read by every CTA after the third cluster barrier
+                }
             }
         }
+        KD_STAMP(7);
         // ------------------------------------------------------------ a4: V rows out, next unit's K rows in behind them
 #pragma unroll 1
         for (int s = 0; s < kTilesPerWarp; ++s) {
@@ -942,16 +1242,22 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
             parity ^= 1u << s;
         }
+        KD_STAMP(8);
         if (kRegRows > 0) {
-            // The register-resident V rows must have ARRIVED, not merely been requested, before any
-            // peer may overwrite their source: fold them into a value the compiler cannot discard.
-            uint32_t fold = 0;
+            // The register-resident V rows must have ARRIVED, not merely been requested, before any peer may
+            // overwrite their source: an empty asm statement that takes the words as inputs makes every one of
+            // those loads complete in front of the barrier's arrive.
 #pragma unroll
             for (int k = 0; k < kRegRows; ++k)
-                fold |= (ra[k].x ^ ra[k].y) ^ (ra[k].z ^ ra[k].w) ^ (rb[k].x ^ rb[k].y) ^ (rb[k].z ^ rb[k].w);
-            if (fold == 0x5bd1e995u && n < 0) atomicExch(p.status, kErrTimeout);   // never true: n > 0
+                asm volatile("" ::"r"(ra[k].x), "r"(ra[k].y), "r"(ra[k].z), "r"(ra[k].w),
+                             "r"(rb[k].x), "r"(rb[k].y), "r"(rb[k].z), "r"(rb[k].w) : "memory");
         }
         cluster_sync_all();   // (3) every warp of the cluster holds the V rows it is responsible for
+        KD_STAMP(9);
+        if (kOnePass && un < p.U) {
+            if (tid < kHeadDim) anchor_from_shares(folded_next, mu_buf + (cur ^ 1) * kHeadDim);
+            __syncthreads();   // the next unit's anchor is complete before any warp scores with it
+        }
         {
             uint4* out = p.v_cache + static_cast<size_t>(u) * N * kRowVec;
 #pragma unroll
@@ -984,9 +1290,34 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 if (lane == 0 && un < p.U) issue_tile(p.k_cache, p.new_k, un, len, B, N, sl, tile, rows_sa, mbar_sa);
             }
         }
-        __syncthreads();   // dst_of is free for the next unit's reduction scratch
+        KD_STAMP(10);
+        if (kOnePass && un < p.U) {
+            // the next unit's tiles, scored by their warp as they land behind the V rows (the first ones have had the
+            // time the later ones took to leave); the key table is free: every CTA has passed the third barrier
+            float2 w[8];
+            const float* mu_next = mu_buf + (cur ^ 1) * kHeadDim;
+            load_anchor(mu_next, t, w);
+            const float m = anchor_norm(mu_next, lane);
+#pragma unroll 1
+            for (int s = 0; s < kTilesPerWarp; ++s) {
+                const int tile = warp + kFusedWarps * s;
+                if (tile >= ntiles) break;
+                mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
+                parity ^= 1u << s;
+                score_tile(rows, tile, rs, t, sub, w, m, p.eps, keys + seg_a);
+            }
+            tiles_scored = true;
+            cur ^= 1;
+            my_share = share_next;
+            folded = folded_next;
+        }
+        KD_STAMP(11);
+        __syncthreads();   // dst_of is free for the next unit
+        KD_STAMP(12);
     }
     cluster_sync_all();   // no CTA leaves while a peer may still address its shared memory
+    KD_STAMP(13);
+    KD_STAMP_FLUSH;
 }
 
 }  // namespace kd

@@ -25,6 +25,21 @@ inline bool cuda_ok(cudaError_t e) {
 #define KD_CUDA(call) do { if (!cuda_ok(call)) return KEYDIFF_ERR_CUDA; } while (0)
 
 constexpr float kDefaultEps = 1e-8f;
+
+// Launch-tuning aids (named in include/keydiff.h): read from the environment ONCE, by keydiff_create; a step
+// never looks at the environment.  A value < 0 means "not set".
+int env_int(const char* name) {
+    const char* v = std::getenv(name);
+    return (v && *v) ? std::atoi(v) : -1;
+}
+
+// Test hook (keydiff_debug_fail_alloc): the n-th device allocation from now on fails once.
+int g_fail_alloc_countdown = 0;
+cudaError_t kd_malloc(void** p, size_t bytes) {
+    if (g_fail_alloc_countdown > 0 && --g_fail_alloc_countdown == 0) { *p = nullptr; return cudaErrorMemoryAllocation; }
+    return cudaMalloc(p, bytes);
+}
+template <typename T> cudaError_t kd_malloc(T** p, size_t bytes) { return kd_malloc(reinterpret_cast<void**>(p), bytes); }
 constexpr int kMaxSelectSmem = 200 * 1024;   // score keys of one unit must fit one CTA
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -48,16 +63,17 @@ struct keydiff_ctx {
     int slot_ring_tiles = 0;    //   fused_smem_bytes, fused_max_clusters describe it)
     int slot_nwords = 0;
     int sm_count = 0;           // SMs of the ctx's device
+    int tune_cluster = -1, tune_stagger_ns = -1, tune_late_ns = -1;   // KEYDIFF_* tuning aids as keydiff_create read them
     // running anchor of the fused path: sum of k/||k|| over the cached rows, per unit
     bool incremental = true;    // use it (one-pass kernel) when it is valid
     bool anchor_valid = false;  // the buffers describe the cache as the last evicting step left it
     int anchor_par = 0;         // which of the two sum buffers the next step reads
     int steps_since_full = 0;   // one-pass steps since the anchor was last recomputed from all rows
     double* anchor_sum[2] = {nullptr, nullptr};   // [U][128]
-    float* anchor_delta = nullptr;                // [U][cluster][128]
+    double* anchor_delta = nullptr;               // [U][cluster][128]
     float eps = kDefaultEps;
     // device scratch
-    float* partial = nullptr;         // [U][splits][128]
+    double* partial = nullptr;        // [U][splits][128]
     float* norms = nullptr;           // [U][nmax]
     float* scores = nullptr;          // [U][nmax]
     int32_t* kept_idx = nullptr;      // [U][N]
@@ -156,8 +172,7 @@ int max_active_clusters(Kernel kern, int C, int smem, int sm_count) {
 bool plan_fused(keydiff_ctx* c, int sm_count) {
     using namespace kd;
     constexpr double kUnitFixedUs = 10.3, kRowUs = 0.0202;
-    int forced = 0;
-    if (const char* env = std::getenv("KEYDIFF_CLUSTER_SIZE")) forced = std::atoi(env);   // tuning aid
+    const int forced = c->tune_cluster;
     double best = 0.0;
     bool found = false;
     for (int C = 1; C <= kMaxCluster; ++C) {
@@ -197,8 +212,7 @@ bool plan_fused(keydiff_ctx* c, int sm_count) {
 bool plan_slot_stream(keydiff_ctx* c, int sm_count) {
     using namespace kd;
     if (c->cfg.max_block > kSlotMaxBlock) return false;
-    int forced = 0;
-    if (const char* env = std::getenv("KEYDIFF_CLUSTER_SIZE")) forced = std::atoi(env);   // tuning aid
+    const int forced = c->tune_cluster;
     const int nwords = (c->nmax + 31) / 32;
     double best = 0.0;
     bool found = false;
@@ -275,8 +289,8 @@ int launch_slot_stream(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, co
             p.late_ns = static_cast<unsigned>(0.5 * unit_ns);
         }
     }
-    if (const char* env = std::getenv("KEYDIFF_STAGGER_NS")) p.stagger_ns = static_cast<unsigned>(std::atoi(env));   // tuning aid
-    if (const char* env = std::getenv("KEYDIFF_LATE_NS")) p.late_ns = static_cast<unsigned>(std::atoi(env));   // tuning aid
+    if (c->tune_stagger_ns >= 0) p.stagger_ns = static_cast<unsigned>(c->tune_stagger_ns);
+    if (c->tune_late_ns >= 0) p.late_ns = static_cast<unsigned>(c->tune_late_ns);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(nclusters * c->cluster);
     cfg.blockDim = dim3(kFusedThreads);
@@ -323,7 +337,7 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
         const double unit_ns = 4.0 * p.rows_per_cta * kRowBytes / 60.0 + 6000.0;
         p.stagger_ns = static_cast<unsigned>(unit_ns / nclusters);
     }
-    if (const char* env = std::getenv("KEYDIFF_STAGGER_NS")) p.stagger_ns = static_cast<unsigned>(std::atoi(env));   // tuning aid
+    if (c->tune_stagger_ns >= 0) p.stagger_ns = static_cast<unsigned>(c->tune_stagger_ns);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(nclusters * c->cluster);
     cfg.blockDim = dim3(kFusedThreads);
@@ -364,9 +378,8 @@ int launch_staged(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const u
 
 }  // namespace
 
-extern "C" {
-
-int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
+namespace {
+int create_impl(const keydiff_config* cfg, keydiff_ctx** out) {
     if (!cfg || !out) return KEYDIFF_ERR_INVALID_ARG;
     if (cfg->n_layers < 1 || cfg->batch < 1 || cfg->n_kv_heads < 1 || cfg->budget < 1 || cfg->max_block < 1 ||
         cfg->device < 0 || cfg->eps < 0.f)
@@ -401,19 +414,22 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
     c->nmax = static_cast<int>(nmax);
     c->eps = cfg->eps > 0.f ? cfg->eps : kDefaultEps;
     c->sm_count = prop.multiProcessorCount;
+    c->tune_cluster = env_int("KEYDIFF_CLUSTER_SIZE");
+    c->tune_stagger_ns = env_int("KEYDIFF_STAGGER_NS");
+    c->tune_late_ns = env_int("KEYDIFF_LATE_NS");
     c->path = KEYDIFF_PATH_STAGED;
     // enough CTAs to fill 148 SMs a few times over, but at least 64 rows per slice
     const int want = (4 * prop.multiProcessorCount + c->U - 1) / c->U;
     c->splits = std::max(1, std::min({want, (c->nmax + 63) / 64, 64}));
 
     bool ok = true;
-    ok = ok && cudaMalloc(&c->partial, sizeof(float) * c->U * c->splits * kd::kHeadDim) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->norms, sizeof(float) * U * nmax) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->scores, sizeof(float) * U * nmax) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->kept_idx, sizeof(int32_t) * U * cfg->budget) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->first_evicted, sizeof(int32_t) * U) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->status, sizeof(int32_t)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->moved_rows, sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && kd_malloc(&c->partial, sizeof(double) * c->U * c->splits * kd::kHeadDim) == cudaSuccess;
+    ok = ok && kd_malloc(&c->norms, sizeof(float) * U * nmax) == cudaSuccess;
+    ok = ok && kd_malloc(&c->scores, sizeof(float) * U * nmax) == cudaSuccess;
+    ok = ok && kd_malloc(&c->kept_idx, sizeof(int32_t) * U * cfg->budget) == cudaSuccess;
+    ok = ok && kd_malloc(&c->first_evicted, sizeof(int32_t) * U) == cudaSuccess;
+    ok = ok && kd_malloc(&c->status, sizeof(int32_t)) == cudaSuccess;
+    ok = ok && kd_malloc(&c->moved_rows, sizeof(unsigned long long)) == cudaSuccess;
     if (ok) {
         ok = cudaMemset(c->scores, 0, sizeof(float) * U * nmax) == cudaSuccess &&
              cudaMemset(c->kept_idx, 0, sizeof(int32_t) * U * cfg->budget) == cudaSuccess &&
@@ -426,7 +442,7 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
                                   kMaxSelectSmem) == cudaSuccess;
     }
     if (ok && cfg->compaction == KEYDIFF_COMPACT_SLOT_REUSE) {
-        ok = cudaMalloc(&c->pos, sizeof(int32_t) * U * cfg->budget) == cudaSuccess &&
+        ok = kd_malloc(&c->pos, sizeof(int32_t) * U * cfg->budget) == cudaSuccess &&
              cudaMemset(c->pos, 0, sizeof(int32_t) * U * cfg->budget) == cudaSuccess &&
              cudaFuncSetAttribute(kd::slot_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   std::max(48 * 1024, 8 * cfg->max_block)) == cudaSuccess;
@@ -438,12 +454,11 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
         if (c->slot_stream || (!slot_reuse(c) && plan_fused(c, prop.multiProcessorCount))) {
             c->path = KEYDIFF_PATH_FUSED;
             const size_t sum_bytes = sizeof(double) * U * kd::kHeadDim;
-            ok = cudaMalloc(&c->anchor_sum[0], sum_bytes) == cudaSuccess && cudaMalloc(&c->anchor_sum[1], sum_bytes) == cudaSuccess &&
-                 cudaMalloc(&c->anchor_delta, sizeof(float) * U * c->cluster * kd::kHeadDim) == cudaSuccess &&
+            ok = kd_malloc(&c->anchor_sum[0], sum_bytes) == cudaSuccess && kd_malloc(&c->anchor_sum[1], sum_bytes) == cudaSuccess &&
+                 kd_malloc(&c->anchor_delta, sizeof(double) * U * c->cluster * kd::kHeadDim) == cudaSuccess &&
                  cudaMemset(c->anchor_sum[0], 0, sum_bytes) == cudaSuccess && cudaMemset(c->anchor_sum[1], 0, sum_bytes) == cudaSuccess &&
-                 cudaMemset(c->anchor_delta, 0, sizeof(float) * U * c->cluster * kd::kHeadDim) == cudaSuccess &&
+                 cudaMemset(c->anchor_delta, 0, sizeof(double) * U * c->cluster * kd::kHeadDim) == cudaSuccess &&
                  cudaDeviceSynchronize() == cudaSuccess;
-            if (const char* env = std::getenv("KEYDIFF_INCREMENTAL")) c->incremental = env[0] != '0';   // tuning aid
         } else if (cfg->path == KEYDIFF_PATH_FUSED) {
             free_scratch(c);
             delete c;
@@ -461,6 +476,15 @@ int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
     cudaSetDevice(prev);
     *out = c;
     return KEYDIFF_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out) {
+    const int rc = create_impl(cfg, out);
+    g_fail_alloc_countdown = 0;   // the test hook serves one keydiff_create
+    return rc;
 }
 
 int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache, const void* new_k, const void* new_v,
@@ -634,6 +658,27 @@ int keydiff_get_positions(const keydiff_ctx* ctx, const int32_t** pos, long long
     return KEYDIFF_OK;
 }
 
+int keydiff_set_positions(keydiff_ctx* ctx, const int32_t* pos_device, int32_t len, long long next_pos, void* stream) {
+    if (!ctx || len < 0 || len > ctx->cfg.budget || next_pos < len || next_pos > 0x7fffffffLL) return KEYDIFF_ERR_INVALID_ARG;
+    if (!slot_reuse(ctx)) return KEYDIFF_ERR_STATE;
+    int dev = -1;
+    KD_CUDA(cudaGetDevice(&dev));
+    if (dev != ctx->cfg.device) return KEYDIFF_ERR_STATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int total = ctx->U * ctx->cfg.budget;
+    if (pos_device) {
+        KD_CUDA(cudaMemcpyAsync(ctx->pos, pos_device, sizeof(int32_t) * total, cudaMemcpyDeviceToDevice, st));
+    } else {
+        kd::pos_iota_kernel<<<(total + 255) / 256, 256, 0, st>>>(ctx->pos, ctx->cfg.budget, total);
+        KD_CUDA(cudaGetLastError());
+    }
+    ctx->len = len;
+    ctx->next_pos = next_pos;
+    ctx->pos_stale = false;
+    ctx->anchor_valid = false;   // the caller brought its own cache contents
+    return KEYDIFF_OK;
+}
+
 int keydiff_get_moved_rows(const keydiff_ctx* ctx, const unsigned long long** counter) {
     if (!ctx || !counter) return KEYDIFF_ERR_INVALID_ARG;
     *counter = ctx->moved_rows;
@@ -663,6 +708,35 @@ const char* keydiff_strerror(int code) {
 }
 
 int keydiff_last_cuda_error(void) { return g_last_cuda_error; }
+
+int keydiff_selftest_bounded_wait(int32_t* status_device, int32_t polls, void* stream) {
+    if (!status_device || polls < 1 || polls > 4096) return KEYDIFF_ERR_INVALID_ARG;
+    kd::bounded_wait_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(status_device, static_cast<uint32_t>(polls));
+    KD_CUDA(cudaGetLastError());
+    return KEYDIFF_OK;
+}
+
+#ifdef KEYDIFF_PHASE_STAMPS
+// Phase-stamp build only: copies the per-CTA, per-phase nanosecond totals of the fused kernel to out_host
+// ([ctas][16] unsigned 64-bit, ctas <= 2368) and optionally clears them.  Synchronises the device.
+__attribute__((visibility("default"))) int keydiff_debug_phase_ns(unsigned long long* out_host, int32_t ctas, int32_t reset) {
+    if (!out_host || ctas < 1 || ctas > kd::kMaxStampCtas) return KEYDIFF_ERR_INVALID_ARG;
+    KD_CUDA(cudaDeviceSynchronize());
+    KD_CUDA(cudaMemcpyFromSymbol(out_host, kd::g_phase_ns, sizeof(unsigned long long) * ctas * kd::kMaxPhases));
+    if (reset) {
+        void* addr = nullptr;
+        KD_CUDA(cudaGetSymbolAddress(&addr, kd::g_phase_ns));
+        KD_CUDA(cudaMemset(addr, 0, sizeof(unsigned long long) * kd::kMaxStampCtas * kd::kMaxPhases));
+    }
+    return KEYDIFF_OK;
+}
+#endif
+
+int keydiff_debug_fail_alloc(int32_t nth) {
+    if (nth < 0) return KEYDIFF_ERR_INVALID_ARG;
+    g_fail_alloc_countdown = nth;
+    return KEYDIFF_OK;
+}
 
 }  // extern "C"
 
@@ -729,6 +803,18 @@ extern "C" int keydiff_evict_static(void* k_cache, void* v_cache, const void* ne
     const uint4* nv = static_cast<const uint4*>(new_v);
     const long long n = static_cast<long long>(len) + block_B;
     const int N = budget_N, U = n_units;
+    // set-up (first call on a device only) comes before anything is enqueued, whatever kind of step this is
+    unsigned char* base = nullptr;
+    const int src = static_scratch_for_current_device(&base);
+    if (src != KEYDIFF_OK) return src;
+    {
+        // the tensors must live on the current device: the scratch address was looked up for it
+        int dev = -1;
+        KD_CUDA(cudaGetDevice(&dev));
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, k_cache) != cudaSuccess) { cudaGetLastError(); return KEYDIFF_ERR_INVALID_ARG; }
+        if (attr.type == cudaMemoryTypeDevice && attr.device != dev) return KEYDIFF_ERR_STATE;
+    }
     if (n <= N) {   // budget not exceeded: plain append, no scratch involved
         const int threads = 256;
         const dim3 grid((block_B * kRowVec + threads - 1) / threads, U, 2);
@@ -742,17 +828,14 @@ extern "C" int keydiff_evict_static(void* k_cache, void* v_cache, const void* ne
     size_t off = 0;
     auto take = [&off](size_t bytes) { const size_t o = off; off += round256(bytes); return o; };
     const size_t o_moved = take(sizeof(unsigned long long));
-    const size_t o_partial = take(sizeof(float) * U * splits * kHeadDim);
+    const size_t o_partial = take(sizeof(double) * U * splits * kHeadDim);
     const size_t o_norms = take(sizeof(float) * U * n);
     const size_t o_scores = take(sizeof(float) * U * n);
     const size_t o_kept = take(sizeof(int32_t) * static_cast<size_t>(U) * N);
     const size_t o_first = take(sizeof(int32_t) * U);
     if (off > kStaticScratchBytes) return KEYDIFF_ERR_TOO_LARGE;
-    unsigned char* base = nullptr;
-    const int src = static_scratch_for_current_device(&base);
-    if (src != KEYDIFF_OK) return src;
     unsigned long long* moved = reinterpret_cast<unsigned long long*>(base + o_moved);
-    float* partial = reinterpret_cast<float*>(base + o_partial);
+    double* partial = reinterpret_cast<double*>(base + o_partial);
     float* norms = reinterpret_cast<float*>(base + o_norms);
     float* scores = reinterpret_cast<float*>(base + o_scores);
     int32_t* kept = reinterpret_cast<int32_t*>(base + o_kept);

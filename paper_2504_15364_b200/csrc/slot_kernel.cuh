@@ -35,7 +35,7 @@ __host__ __device__ inline SlotLayout slot_layout(int ring_tiles, int nkeys, int
     int off = 0;
     auto take = [&off](int bytes) { const int o = off; off += (bytes + 127) & ~127; return o; };
     L.ring = take(ring_tiles * kTileRows * kRowBytes);
-    L.keys = take(nkeys * 4 > kBins * 4 ? nkeys * 4 : kBins * 4);   // also 8 KB of reduction scratch while the table is dead
+    L.keys = take(nkeys * 4 > kReduceBytes ? nkeys * 4 : kReduceBytes);   // also the reduction scratch while the table is dead
     L.work = take(kBins * 4);            // warp-reduction scratch / histogram
     L.bitmap = take(2 * nwords * 4);     // evicted-candidate bitmap, evicted-before count of every word
     L.cand = take(2 * kCandCap * 4);     // keys and indices of the threshold bin
@@ -63,7 +63,7 @@ struct SlotParams {
     unsigned late_ns;      // clusters that serve one unit fewer than the others start this much later still
     float* scores; int32_t* kept_idx; int32_t* first_evicted;
     unsigned long long* moved_rows; int32_t* status;
-    const double* anchor_in; double* anchor_out; float* anchor_delta;   // running anchor, as in FusedParams
+    const double* anchor_in; double* anchor_out; double* anchor_delta;   // running anchor, as in FusedParams
     int raw_anchor, window;
     int32_t* pos;       // [U][N] token position of every slot
     int next_pos;       // position of the block's first token
@@ -83,6 +83,18 @@ __device__ __forceinline__ void issue_rows(const uint4* cache, const uint4* bloc
                   block + (static_cast<size_t>(u) * B + (g0 + from_cache - len)) * kRowVec, from_block * kRowBytes, bar);
 }
 
+// Row j of a CTA's share of a list of candidate numbers: entry (j / 64) * step + base + j % 64 of the list (the
+// share is every `step / 64`-th run of 64 entries), as a pointer to that candidate's key row.  A list entry
+// outside [0, n) cannot occur; the clamp makes sure that even then no address outside the tensors is formed.
+struct ListedRows {
+    const uint4* cache; const uint4* block; const int* list;
+    int u, len, B, N, n, step, base;
+    __device__ __forceinline__ const uint4* operator()(int j) const {
+        const int v = list[(j / kGroups) * step + base + (j % kGroups)];
+        return concat_row(cache, block, u, min(max(v, 0), n - 1), len, B, N);
+    }
+};
+
 __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const SlotParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int C = p.cluster;
@@ -90,7 +102,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
     const uint4* ring = reinterpret_cast<const uint4*>(smem + L.ring);
     uint32_t* keys = reinterpret_cast<uint32_t*>(smem + L.keys);
     int* hist = reinterpret_cast<int*>(smem + L.work);
-    float* red = reinterpret_cast<float*>(smem + L.work);
     uint32_t* bitmap = reinterpret_cast<uint32_t*>(smem + L.bitmap);
     int* wlocal = reinterpret_cast<int*>(smem + L.bitmap) + p.nwords;
     uint32_t* cand_key = reinterpret_cast<uint32_t*>(smem + L.cand);
@@ -156,58 +167,38 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
 
     for (int u = cluster_id; u < p.U; u += nclusters) {
         const int un = u + nclusters;
-        float block_sum = 0.f;   // tid < 128: channel tid of the block rows' sum of k/||k||
+        double block_sum = 0.0;   // tid < 128: channel tid of the block rows' sum of k/||k||
         // ------------------------------------------------------------ anchor from the running sum + the block rows
         {
             double run = 0.0;
-            float dl[kMaxCluster];
+            double dl[kMaxCluster];
             if (tid < kHeadDim) {
                 run = p.anchor_in[static_cast<size_t>(u) * kHeadDim + tid];
 #pragma unroll
                 for (int c = 0; c < kMaxCluster; ++c)
-                    dl[c] = c < C ? p.anchor_delta[(static_cast<size_t>(u) * C + c) * kHeadDim + tid] : 0.f;
+                    dl[c] = c < C ? p.anchor_delta[(static_cast<size_t>(u) * C + c) * kHeadDim + tid] : 0.0;
             }
-            float2 acc[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) acc[q] = make_float2(0.f, 0.f);
-            for (int b0 = 0; b0 < B; b0 += kGroups) {   // (same trip count in every lane: row_a1 shuffles)
-                const int br = b0 + g;
-                uint4 a = make_uint4(0, 0, 0, 0), b = a;
-                if (br < B) {
-                    const uint4* row = p.new_k + (static_cast<size_t>(u) * B + br) * kRowVec;
-                    a = row[t]; b = row[t + 8];
-                }
-                row_a1(a, b, br < B, inv_eps, acc, raw);
+            // every CTA normalises the whole block itself; scratch: the work area (the key table cannot lend its space
+            // here: a peer that is ahead may already be pushing its keys of this unit into it)
+            {
+                const ContiguousRows blk{p.new_k + static_cast<size_t>(u) * B * kRowVec};
+                block_sum = global_rows_terms_sum(blk, B, inv_eps, raw,
+                                                  reinterpret_cast<float*>(smem + L.work) + 8 * kHeadDim,
+                                                  reinterpret_cast<double*>(smem + L.work), tid);
             }
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                float2 v = acc[q];
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
-                acc[q] = v;
-            }
-            if (lane < 8) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    *reinterpret_cast<float2*>(&red[warp * kHeadDim + lane_channel(t, 2 * q)]) = acc[q];
-            }
-            __syncthreads();
             if (tid < kHeadDim) {
-#pragma unroll
-                for (int w = 0; w < kFusedWarps; ++w) block_sum += red[w * kHeadDim + tid];
                 double a = run;
 #pragma unroll
-                for (int c = 0; c < kMaxCluster; ++c) a += static_cast<double>(dl[c]);   // rank order; absent ranks add 0
+                for (int c = 0; c < kMaxCluster; ++c) a += dl[c];   // rank order; absent ranks add 0
                 if (crank == 0) p.anchor_out[static_cast<size_t>(u) * kHeadDim + tid] = a;   // the cached rows' sum, folded
-                mu_sh[tid] = static_cast<float>((a + static_cast<double>(block_sum)) / static_cast<double>(n));
+                mu_sh[tid] = static_cast<float>((a + block_sum) / static_cast<double>(n));
             }
             __syncthreads();
         }
         // ------------------------------------------------------------ a1 + a2 in one pass over the stream
         {
             float2 w[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) w[q] = *reinterpret_cast<const float2*>(&mu_sh[lane_channel(t, 2 * q)]);
+            load_anchor(mu_sh, t, w);
             float m;   // ||mu||, computed by every warp in the same order
             {
                 const float4 c4 = reinterpret_cast<const float4*>(mu_sh)[lane];
@@ -224,15 +215,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
                 c_par ^= 1u << c_d;
                 const int lo = (warp + kFusedWarps * j) * kTileRows;   // first slice row of the tile
                 const uint4* tile = ring + phys * kTileRows * kRowVec;
-                float v[8];   // this lane's shares of the tile's four rows of its row group
+                float vs[4];   // this lane's shares of the tile's four rows of its row group
+                double vd[4];
 #pragma unroll
                 for (int it = 0; it < 4; ++it) {
                     const int r = it * 4 + sub;
                     uint4 a = make_uint4(0, 0, 0, 0), b = a;
                     if (lo + r < seg) { a = tile[r * kRowVec + t]; b = tile[r * kRowVec + t + 8]; }
-                    lane_sumsq_dot(a, b, w, v[2 * it], v[2 * it + 1]);
+                    lane_sumsq_dot(a, b, w, vs[it], vd[it]);
                 }
-                const uint32_t key = score4(v, t, m, p.eps);
+                const uint32_t key = score4(vs, vd, t, m, p.eps);
                 const int lr = lo + (t >> 1) * 4 + sub;
                 if (!(t & 1) && lr < seg) {
                     keys[seg_a + lr] = key;
@@ -274,91 +266,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
             __syncthreads();
         }
         // ------------------------------------------------------------ a3: the bitmap of evicted candidates
-        bool planned = false;
+        // the low-end select of fused_kernel.cuh; ties: (key ascending, candidate number descending) go first
         int* wbase = sel.hist + 2 * kFusedWarps;
-        if (fast_ok) {
-            // the low-end select of fused_kernel.cuh: keys in registers, 2048 bins over the low end of the unit's
-            // own key range, candidates under the threshold bin straight into the bitmap, the bin's own keys
-            // ranked exactly under (key ascending, candidate number descending)
-            uint32_t* wmin = reinterpret_cast<uint32_t*>(sel.hist);
-            uint32_t* wmax = reinterpret_cast<uint32_t*>(sel.hist) + kFusedWarps;
-            const int cnt = (n - tid + kFusedThreads - 1) / kFusedThreads;
-            uint32_t kk[kFastKeys];
-#pragma unroll
-            for (int j = 0; j < kFastKeys; ++j) kk[j] = j < cnt ? keys[tid + j * kFusedThreads] : 0xffffffffu;
-            {
-                uint32_t lo = 0xffffffffu, hi = 0u;
-#pragma unroll
-                for (int j = 0; j < kFastKeys; ++j) { lo = min(lo, kk[j]); if (j < cnt) hi = max(hi, kk[j]); }
-                const uint32_t cut = (n >= kFusedThreads && E <= kFusedThreads) ? lo : hi;   // bounds the E-th smallest key
-                const uint32_t wlo = __reduce_min_sync(0xffffffffu, lo);
-                const uint32_t wcut = __reduce_max_sync(0xffffffffu, cnt > 0 ? cut : 0u);
-                if (lane == 0) { wmin[warp] = wlo; wmax[warp] = wcut; }
-            }
-            __syncthreads();
-            uint32_t kmin, kcut, shift;
-            {
-                const uint32_t lo = lane < kFusedWarps ? wmin[lane] : 0xffffffffu, hi = lane < kFusedWarps ? wmax[lane] : 0u;
-                kmin = __reduce_min_sync(0xffffffffu, lo);
-                kcut = __reduce_max_sync(0xffffffffu, hi);
-                const int bits = 32 - __clz(kcut - kmin);
-                shift = bits > 11 ? bits - 11 : 0;
-            }
-            auto bin_of = [kmin, kcut, shift](uint32_t k) { return k <= kcut ? min((k - kmin) >> shift, 2046u) : 2047u; };
-#pragma unroll
-            for (int j = 0; j < kFastKeys; ++j) {
-                // (the top bin holds every key above the bound: the crossing is never there, so it is not counted)
-                const uint32_t b = bin_of(kk[j]);
-                if (j < cnt && b != 2047u) atomicAdd(&hist[b], 1);
-            }
-            __syncthreads();
-            const int packed = find_crossing(hist, E, lane, warp, sel.warp_eq);
-            const uint32_t bstar = static_cast<uint32_t>(packed >> 16);
-            const int need = E - (packed & 0xffff);   // this many keys of the threshold bin go
-            unsigned m_below = 0, m_in = 0;
-#pragma unroll
-            for (int j = 0; j < kFastKeys; ++j) {
-                const uint32_t b = bin_of(kk[j]);
-                m_below |= (j < cnt && b < bstar) ? 1u << j : 0u;
-                m_in |= (j < cnt && b == bstar) ? 1u << j : 0u;
-            }
-            {
-                int first = n;
-                if (packed >= 0 && (m_below | m_in)) {
-                    for (unsigned mm = m_below; mm; mm &= mm - 1) {
-                        const int i = tid + (__ffs(mm) - 1) * kFusedThreads;
-                        atomicOr(&bitmap[i >> 5], 1u << (i & 31));
-                        first = min(first, i);
-                    }
-                    for (unsigned mm = m_in; mm; mm &= mm - 1) {
-                        const int i = tid + (__ffs(mm) - 1) * kFusedThreads;
-                        const int slot = atomicAdd(&misc[0], 1);
-                        if (slot < kFastCandCap) { cand_key[slot] = keys[i]; cand_idx[slot] = i; }
-                    }
-                }
-                first = __reduce_min_sync(0xffffffffu, first);   // one shared-memory atomic per warp, not per thread
-                if (lane == 0 && first < n) atomicMin(&misc[1], first);
-            }
-            __syncthreads();
-            const int ncand = misc[0];
-            if (packed >= 0 && ncand <= kFastCandCap) {   // uniform: every thread sees the same values
-                int wfirst = n;
-                for (int c = warp; c < ncand; c += kFusedWarps) {
-                    const uint32_t mk = cand_key[c];
-                    const int mi = cand_idx[c];
-                    int rank = 0;
-                    for (int q = lane; q < ncand; q += 32) {
-                        const uint32_t ok = cand_key[q];
-                        rank += (ok < mk) || (ok == mk && cand_idx[q] > mi);
-                    }
-                    rank = __reduce_add_sync(0xffffffffu, rank);
-                    if (lane == 0 && rank < need) { atomicOr(&bitmap[mi >> 5], 1u << (mi & 31)); wfirst = min(wfirst, mi); }
-                }
-                if (lane == 0 && wfirst < n) atomicMin(&misc[1], wfirst);
-                planned = true;
-            }
-            __syncthreads();
-        }
+        const bool planned = fast_ok && low_end_select(keys, n, E, hist, bitmap, cand_key, cand_idx, sel, misc);
         if (!planned) {
             // the full-table select writes the same bitmap (cleared first: the attempt above may have marked some)
             for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;
@@ -429,27 +339,23 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
         __syncthreads();
         // ------------------------------------------------------------ a4: evicted rows leave the running sum, kept block rows take the freed slots
         {
-            float2 gone[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) gone[q] = make_float2(0.f, 0.f);
-            // (a) evicted rows, read once more (from L2); the next row is requested before this one is used
+            // (a) evicted rows, read once more (from L2): their terms leave the running sum.  The CTA that re-reads
+            // evicted row r is the one that overwrites its slot in (b): rows r with (r / 64) % C == crank.
             const int stride = C * kGroups, r_first = crank * kGroups + g;
-            uint4 na = make_uint4(0, 0, 0, 0), nb = na;
-            if (r_first < E) {
-                const uint4* row = concat_row(p.k_cache, p.new_k, u, ev_of[r_first], len, B, N);
-                na = row[t]; nb = row[t + 8];
+            double gone = 0.0;   // tid < 128: channel tid of this CTA's evicted rows' sum of terms
+            {
+                const int rem = E % stride - crank * kGroups;
+                const int mine = (E / stride) * kGroups + min(max(rem, 0), kGroups);
+                const uint4* kc = p.k_cache; const uint4* nk = p.new_k;
+                float* inv_sh = reinterpret_cast<float*>(keys);   // the key table is dead until the next unit
+                const ListedRows rows_of{kc, nk, ev_of, u, len, B, N, n, stride, crank * kGroups};
+                gone = global_rows_terms_sum(rows_of, mine, inv_eps, raw, inv_sh, reinterpret_cast<double*>(inv_sh + kHeadDim), tid);
+                if (tid < kHeadDim)
+                    p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (crank == 0 ? block_sum : 0.0) - gone;
+                __syncthreads();   // every evicted row of this CTA's share has been read: its slot may be overwritten
             }
-            for (int r0 = 0; r0 < E; r0 += stride) {   // (same trip count in every lane: row_a1 shuffles)
-                const int r = r0 + r_first;
-                const uint4 a = na, b = nb;
-                if (r + stride < E) {
-                    const uint4* row = concat_row(p.k_cache, p.new_k, u, ev_of[r + stride], len, B, N);
-                    na = row[t]; nb = row[t + 8];
-                }
-                row_a1(a, b, r < E, inv_eps, gone, raw);   // (a row past the end is all zeros and is not added)
-            }
-            // (b) kept block row r into freed slot r.  For r < evicted_cache that slot is evicted row r, whose
-            // old words the same lanes read in (a): a lane's own load and store to one address stay in order.
+            // (b) kept block row r into freed slot r.  For r < evicted_cache that slot is evicted row r, which this
+            // same CTA re-read in (a), in front of the barrier above.
 #pragma unroll 2
             for (int r = r_first; r < kb; r += stride) {
                 const int slot = slot_of[r], j = blk_of[r];
@@ -465,26 +371,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
                     if (p.kept_mirror) p.kept_mirror[static_cast<size_t>(u) * N + slot] = len + j;
                     p.pos[static_cast<size_t>(u) * N + slot] = p.next_pos + j;
                 }
-            }
-            float* red2 = reinterpret_cast<float*>(keys);   // the key table is dead until the next unit
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                float2 v = gone[q];
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 8);  v.y += __shfl_xor_sync(0xffffffffu, v.y, 8);
-                v.x += __shfl_xor_sync(0xffffffffu, v.x, 16); v.y += __shfl_xor_sync(0xffffffffu, v.y, 16);
-                gone[q] = v;
-            }
-            if (lane < 8) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    *reinterpret_cast<float2*>(&red2[warp * kHeadDim + lane_channel(t, 2 * q)]) = gone[q];
-            }
-            __syncthreads();
-            if (tid < kHeadDim) {
-                float e = 0.f;
-#pragma unroll
-                for (int w = 0; w < kFusedWarps; ++w) e += red2[w * kHeadDim + tid];
-                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (crank == 0 ? block_sum : 0.f) - e;
             }
         }
         if (C > 1) { cluster_arrive(); exchange_pending = true; }   // this CTA is done with the unit's key table

@@ -24,15 +24,19 @@ __device__ __forceinline__ const uint4* concat_row(const uint4* cache, const uin
 __global__ void __launch_bounds__(kStagedThreads)
 anchor_partial_kernel(const uint4* __restrict__ k_cache, const uint4* __restrict__ new_k,
                       int len, int B, int N, float eps, int rows_per_split, int nmax,
-                      float* __restrict__ partial, float* __restrict__ norms, int raw_anchor) {
-    __shared__ float red[kStagedThreads / kLanesPerRow][kHeadDim + 4];
+                      double* __restrict__ partial, float* __restrict__ norms, int raw_anchor) {
+    __shared__ double red[kStagedThreads / kLanesPerRow][kHeadDim + 2];
     const int u = blockIdx.y, s = blockIdx.x, splits = gridDim.x;
     const int n = len + B;
     const int r0 = s * rows_per_split, r1 = min(n, r0 + rows_per_split);
     const int g = threadIdx.x >> 3, t = threadIdx.x & 7;
+    // a thread adds four rows in fp32, then carries the sums on in double: the anchor is a sum of thousands of
+    // unit vectors that cancels when the keys point in many directions
+    double wide[16];
     float acc[16];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+    for (int j = 0; j < 16; ++j) { wide[j] = 0.0; acc[j] = 0.f; }
+    int pending = 0;
     for (int base = r0; base < r1; base += kStagedThreads / kLanesPerRow) {
         const int i = base + g;
         const bool valid = i < r1;
@@ -50,12 +54,17 @@ anchor_partial_kernel(const uint4* __restrict__ k_cache, const uint4* __restrict
             for (int j = 0; j < 16; ++j) acc[j] = fmaf(x[j], inv, acc[j]);
             if (t == 0) norms[static_cast<size_t>(u) * nmax + i] = r;
         }
+        if (++pending == 4) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) { wide[j] += static_cast<double>(acc[j]); acc[j] = 0.f; }
+            pending = 0;
+        }
     }
 #pragma unroll
-    for (int j = 0; j < 16; ++j) red[g][lane_channel(t, j)] = acc[j];
+    for (int j = 0; j < 16; ++j) red[g][lane_channel(t, j)] = wide[j] + static_cast<double>(acc[j]);
     __syncthreads();
     if (threadIdx.x < kHeadDim) {
-        float sum = 0.f;
+        double sum = 0.0;
         for (int q = 0; q < kStagedThreads / kLanesPerRow; ++q) sum += red[q][threadIdx.x];   // fixed order
         partial[(static_cast<size_t>(u) * splits + s) * kHeadDim + threadIdx.x] = sum;
     }
@@ -66,16 +75,16 @@ anchor_partial_kernel(const uint4* __restrict__ k_cache, const uint4* __restrict
 __global__ void __launch_bounds__(kStagedThreads)
 score_kernel(const uint4* __restrict__ k_cache, const uint4* __restrict__ new_k,
              int len, int B, int N, float eps, int rows_per_split, int nmax,
-             const float* __restrict__ partial, const float* __restrict__ norms,
+             const double* __restrict__ partial, const float* __restrict__ norms,
              float* __restrict__ scores) {
     __shared__ float mu_sh[kHeadDim];
     __shared__ float m_sh;
     const int u = blockIdx.y, s = blockIdx.x, splits = gridDim.x;
     const int n = len + B;
     if (threadIdx.x < kHeadDim) {
-        float sum = 0.f;
+        double sum = 0.0;
         for (int q = 0; q < splits; ++q) sum += partial[(static_cast<size_t>(u) * splits + q) * kHeadDim + threadIdx.x];
-        mu_sh[threadIdx.x] = sum / static_cast<float>(n);
+        mu_sh[threadIdx.x] = static_cast<float>(sum / static_cast<double>(n));
     }
     __syncthreads();
     if (threadIdx.x < 32) {
@@ -239,13 +248,13 @@ slot_place_kernel(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
 
 // Running anchor of the cached rows from the partial sums of anchor_partial_kernel run over the cache
 // alone: sum[u][c] = sum over splits (double), and the pending deltas are cleared.  grid = U, 128 threads.
-__global__ void anchor_fold_kernel(const float* __restrict__ partial, int splits, double* __restrict__ sum,
-                                   float* __restrict__ delta, int ranks) {
+__global__ void anchor_fold_kernel(const double* __restrict__ partial, int splits, double* __restrict__ sum,
+                                   double* __restrict__ delta, int ranks) {
     const int u = blockIdx.x, c = threadIdx.x;
     double a = 0.0;
-    for (int s = 0; s < splits; ++s) a += static_cast<double>(partial[(static_cast<size_t>(u) * splits + s) * kHeadDim + c]);
+    for (int s = 0; s < splits; ++s) a += partial[(static_cast<size_t>(u) * splits + s) * kHeadDim + c];
     sum[static_cast<size_t>(u) * kHeadDim + c] = a;
-    for (int r = 0; r < ranks; ++r) delta[(static_cast<size_t>(u) * ranks + r) * kHeadDim + c] = 0.f;
+    for (int r = 0; r < ranks; ++r) delta[(static_cast<size_t>(u) * ranks + r) * kHeadDim + c] = 0.0;
 }
 
 // Token positions of the slots: identity (a cache the caller filled in token order) ...

@@ -62,11 +62,14 @@ def test_agrees_with_rebuilding_every_step_and_is_deterministic():
         runs.append((k_cache.clone(), v_cache.clone(), kd.scratch()["scores"].clone()))
         kd.close()
     assert all(torch.equal(a, b) for a, b in zip(runs[0], runs[1])), "two runs on the running sum differ"
-    # against the rebuild mode: same cache unless a token sat inside the tolerance band of a threshold
-    same_rows = (runs[0][0] == runs[2][0]).all(dim=2).float().mean().item()
-    assert same_rows > 0.98
+    # against the rebuild mode: same cache unless a token sat inside the tolerance band of a threshold ...
+    same_unit = (runs[0][0] == runs[2][0]).all(dim=2).all(dim=1)
+    assert (runs[0][0] == runs[2][0]).all(dim=2).float().mean().item() > 0.98
+    assert same_unit.float().mean().item() >= 0.5, "most units should never meet a band decision in 40 steps"
+    # ... and on the units whose caches are still identical (the last step scored the same rows) the two
+    # modes' scores agree to 2e-5
     n = wl.budget + wl.block
-    assert torch.allclose(runs[0][2][:, :n], runs[2][2][:, :n], rtol=0, atol=2e-5) or same_rows < 1.0
+    assert torch.allclose(runs[0][2][same_unit, :n], runs[2][2][same_unit, :n], rtol=0, atol=2e-5)
 
 
 def test_set_len_after_outside_changes_rebuilds_the_sum():
