@@ -52,7 +52,7 @@ constexpr int kCandCap = kFusedThreads;                 // exact-rank stage hand
 constexpr int kMaxCluster = 16;
 constexpr int kFastKeys = 17;                           // fast select: keys per thread held in registers (n <= 8704)
 constexpr int kFastCandCap = 192;                       // fast select: keys of the threshold bin ranked exactly
-constexpr int kReduceBytes = 28 * 1024;   // scratch the dead key table lends: staged row terms (16 KB), quarter sums, lists
+constexpr int kReduceBytes = 32 * 1024;   // scratch the dead key table lends: staged row terms (16 KB), quarter sums, lists
 constexpr int kSmemLimit = 232448;                      // opt-in shared memory per CTA on sm_100
 constexpr int kErrTimeout = -6;                         // KEYDIFF_ERR_TIMEOUT
 constexpr uint32_t kWaitSpins = 1u << 24;               // bound of every mbarrier wait
@@ -732,6 +732,37 @@ __device__ __forceinline__ void score_tile(const uint4* rows, int tile, int rs, 
     if (!(t & 1) && lr < rs) keys_seg[lr] = key;   // (both lanes of a pair hold the row's key)
 }
 
+// The canonical form of a row's anchor terms inside the fused kernel: ONE WARP PER ROW, lane l holding channels
+// 4l .. 4l+3 (two packed words).  ||k||^2 = the lanes' four-term chains added by the xor butterfly 16, 8, 4, 2, 1;
+// 1/||k|| by the approximate reciprocal square root (or min with 1/eps); the four terms are the fp32 products,
+// added to acc in double.  Every place that adds or removes a row's terms uses this function, so that a row takes
+// away exactly what it brought.  The whole warp calls; `active` is warp-uniform.
+__device__ __forceinline__ void warp_row_terms(uint2 wds, bool active, float inv_eps, bool raw, double (&acc)[4]) {
+    const float x0 = bf16_lo(wds.x), x1 = bf16_hi(wds.x), x2 = bf16_lo(wds.y), x3 = bf16_hi(wds.y);
+    float ss = fmaf(x3, x3, fmaf(x2, x2, fmaf(x1, x1, x0 * x0)));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (active) {
+        const float inv = raw ? 1.0f : fminf(approx_rsqrt(ss), inv_eps);
+        acc[0] += static_cast<double>(__fmul_rn(x0, inv)); acc[1] += static_cast<double>(__fmul_rn(x1, inv));
+        acc[2] += static_cast<double>(__fmul_rn(x2, inv)); acc[3] += static_cast<double>(__fmul_rn(x3, inv));
+    }
+}
+// A warp's four sums per lane (channels 4l .. 4l+3) into its row of a [16 warps][128] table of doubles.
+__device__ __forceinline__ void store_warp_sums(const double (&acc)[4], double* table, int warp, int lane) {
+    double2* row = reinterpret_cast<double2*>(table + warp * kHeadDim + 4 * lane);
+    row[0] = make_double2(acc[0], acc[1]);
+    row[1] = make_double2(acc[2], acc[3]);
+}
+// Channel c's total over the 16 warps, in warp order.
+__device__ __forceinline__ double sum_warp_sums(const double* table, int c) {
+    double s = 0.0;
+#pragma unroll
+    for (int w = 0; w < kFusedWarps; ++w) s += table[w * kHeadDim + c];
+    return s;
+}
+constexpr int kPreRows = 2;   // block rows per warp and kind requested before the K stores (the rest after them)
+
 // kRegRows = rows per row group that live in registers (the host picks the smallest instance that
 // holds a slice together with the shared-memory rows).
 //
@@ -766,18 +797,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     const uint32_t rows_sa = smem_addr(rows), mbar_sa = smem_addr(smem + L.mbar);
     const uint32_t keys_sa = smem_addr(keys), partials_sa = smem_addr(partials);
     // scratch that the dead key table lends between the selection and the third cluster barrier (no peer writes the
-    // table in that window).  Either the evicted cache rows of the slice are stashed as they are (the K stores put
-    // them there) and turned into terms while the V rows arrive, or -- more of them than the stash holds -- their
-    // terms are staged in rounds before the K stores.
-    uint4* stash = reinterpret_cast<uint4*>(keys);                                     // [kStashRows][16]
-    float* inv_st = reinterpret_cast<float*>(stash + kStashRows * kRowVec);            // [kStashRows]
-    float* inv_ev = inv_st + kStashRows;                                               // [128] evicted block rows of this CTA's range
-    float* inv_nx = inv_ev + kHeadDim;                                                 // [128] the next unit's block rows of that range
-    double* part_g = reinterpret_cast<double*>(inv_nx + kHeadDim);                     // [4][128]
-    double* part_n = part_g + 4 * kHeadDim;                                            // [4][128]
-    float* staged = reinterpret_cast<float*>(keys);                                    // [kTermRows][128]  (rounds only)
-    double* part_gone = reinterpret_cast<double*>(staged + kTermRows * kHeadDim);      // [4][128]
-    int* ev_round = reinterpret_cast<int*>(part_gone + 4 * kHeadDim);                  // [kTermRows]
+    // table in that window): every warp's sums of the terms that left and of the next block's terms
+    double* gone_tab = reinterpret_cast<double*>(keys);                 // [16][128]
+    double* next_tab = gone_tab + kFusedWarps * kHeadDim;               // [16][128]
+    uint4* warp_row = reinterpret_cast<uint4*>(smem + L.xchg);          // [16 warps][16 words]: a register-resident row, re-read
+                                                                        // one warp per row (the candidates' area, dead by then)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = tid >> 3, t = tid & 7, sub = lane >> 3;
     const int crank = static_cast<int>(cluster_ctarank());
@@ -841,7 +865,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     const int b_per = (B + C - 1) / C;
     const int b_lo = min(B, crank * b_per), b_hi = min(B, b_lo + b_per), nb = b_hi - b_lo;
     double my_share = 0.0;       // tid < 128: channel tid of this CTA's share of this unit's block sum
-    double folded = 0.0;         // tid < 128: channel tid of this unit's folded running sum (cached rows)
     bool tiles_scored = false;   // this unit's tiles were scored behind the previous unit's V rows
     int cur = 0;                 // which of the two anchor buffers holds this unit's anchor
     auto fold_running_sum = [&](int uu) -> double {   // threads tid < 128
@@ -865,10 +888,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         mu_out[tid] = static_cast<float>((a + bs) / static_cast<double>(n));
     };
     if (kOnePass && cluster_id < p.U) {   // the first unit's anchor (the work area is free before the first unit)
+        double folded = 0.0;
         if (tid < kHeadDim) folded = fold_running_sum(cluster_id);
-        const ContiguousRows blk{p.new_k + (static_cast<size_t>(cluster_id) * B + b_lo) * kRowVec};
-        my_share = global_rows_terms_sum(blk, nb, inv_eps, raw, reinterpret_cast<float*>(smem + L.work) + 8 * kHeadDim,
-                                         reinterpret_cast<double*>(smem + L.work), tid);
+        {
+            double acc[4] = {0.0, 0.0, 0.0, 0.0};
+            const uint4* blk = p.new_k + static_cast<size_t>(cluster_id) * B * kRowVec;
+            for (int j = b_lo + warp; j < b_hi; j += kFusedWarps)   // (warp-uniform)
+                warp_row_terms(reinterpret_cast<const uint2*>(blk + static_cast<size_t>(j) * kRowVec)[lane], true, inv_eps, raw, acc);
+            store_warp_sums(acc, gone_tab, warp, lane);   // (nobody uses the key table before the first unit's scores)
+            __syncthreads();
+            if (tid < kHeadDim) my_share = sum_warp_sums(gone_tab, tid);
+            __syncthreads();   // the table is free again before any key is written
+        }
         if (tid < kHeadDim) push_share(my_share);
         cluster_sync_all();
         if (tid < kHeadDim) anchor_from_shares(folded, mu_buf);
@@ -1062,53 +1093,27 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             }
         }
         KD_STAMP(4);
-        // ------------------------------------------------------------ the evicted rows leave the running anchor sum
+        // ------------------------------------------------------------ a4: K rows out, V rows in behind them; the rows that leave
+        // the cache and this CTA's range of the next block turn into anchor terms along the way
         // This CTA's delta to the running sum: its share of the block that came in (one-pass steps) minus the terms
-        // of (a) the evicted cache rows of its slice, which only exist on chip once the K stores have run, and (b)
-        // the evicted block rows of its range of the block, which stay readable in global memory.
-        auto evicted_before = [&](int i) { const int w = i >> 5; return wlocal[w] + __popc(bitmap[w] & ((1u << (i & 31)) - 1u)); };
-        const int c_lo = min(seg_a, len), c_hi = min(seg_b, len);             // the slice's cache rows
-        const int eb_lo = evicted_before(c_lo);                               // (len < n: the index is inside the bitmap)
-        const int n_gone_cache = evicted_before(c_hi) - eb_lo;
-        const bool use_stash = n_gone_cache <= kStashRows;
-        double gone_rounds = 0.0;   // tid < 128 after the rounds
-        if (!use_stash) {
-            // Rounds before the K stores: evicted cache row number j of the slice (ascending) is staged as 128
-            // terms in row j of a round of kTermRows rows.
-            double acc = 0.0;
-            const int w_first = c_lo >> 5;
-            for (int r0 = 0; r0 < n_gone_cache; r0 += kTermRows) {
-                const int cnt = min(kTermRows, n_gone_cache - r0);
-                if (r0 > 0) __syncthreads();   // the previous round's terms and list have been read
-                // which staged row is which local row: one thread per bitmap word (-1: the row lives in registers)
-                if (w_first + tid < nwords && ((w_first + tid) << 5) < c_hi) {
-                    const int w = w_first + tid;
-                    int j = wlocal[w] - eb_lo - r0;
-                    for (uint32_t wd = bitmap[w]; wd; wd &= wd - 1, ++j) {
-                        const int i = 32 * w + __ffs(wd) - 1;
-                        if (i >= c_lo && i < c_hi && j >= 0 && j < kTermRows) ev_round[j] = i - seg_a < rs ? i - seg_a : -1;
-                    }
-                }
+        // of (a) the evicted cache rows of its slice -- each taken by the warp that holds it, from the tile or the
+        // registers, just before the K stores hand the tile on -- and (b) the evicted block rows of its range of the
+        // block, which stay readable in global memory (warp w takes rows w, w + 16, ... of the range).
+        double acc_g[4] = {0.0, 0.0, 0.0, 0.0}, acc_n[4] = {0.0, 0.0, 0.0, 0.0};
+        const bool next_share = kOnePass && un < p.U;
+        const uint4* blk_u = p.new_k + static_cast<size_t>(u) * B * kRowVec;
+        const uint4* blk_n = p.new_k + static_cast<size_t>(next_share ? un : u) * B * kRowVec;
+        auto block_row_evicted = [&](int j) { const int i = len + j; return j < b_hi && ((bitmap[i >> 5] >> (i & 31)) & 1u) != 0; };
+        uint2 pre_e[kPreRows], pre_n[kPreRows];   // requested now, used after the K stores
 #pragma unroll
-                for (int k = 0; k < kRegRows; ++k) {   // register-resident rows: their own row group
-                    const int lr = rs + k * kGroups + g;
-                    const int j = (lr < seg && seg_a + lr < len && dst_of[lr] < 0) ? evicted_before(seg_a + lr) - eb_lo - r0 : -1;
-                    row_terms(ra[k], rb[k], t, inv_eps, raw, j >= 0 && j < kTermRows, staged + max(j, 0) * kHeadDim);
-                }
-                __syncthreads();
-                if (g < kTermRows) {   // (warps 0..7, warp-uniform: row_terms shuffles) row group g takes staged row g
-                    const int lr = g < cnt ? ev_round[g] : -1;
-                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
-                    if (lr >= 0) { a = rows[lr * kRowVec + t]; b = rows[lr * kRowVec + t + 8]; }
-                    row_terms(a, b, t, inv_eps, raw, lr >= 0, staged + g * kHeadDim);
-                }
-                __syncthreads();
-                terms_sum(staged, cnt, tid, acc);
-            }
-            gone_rounds = quarters_sum(acc, part_gone, tid);
-            __syncthreads();   // the scratch is free for what follows
+        for (int k = 0; k < kPreRows; ++k) {
+            const int j = b_lo + warp + k * kFusedWarps;
+            pre_e[k] = make_uint2(0, 0); pre_n[k] = pre_e[k];
+            if (block_row_evicted(j)) pre_e[k] = reinterpret_cast<const uint2*>(blk_u + static_cast<size_t>(j) * kRowVec)[lane];
+            if (next_share && j < b_hi) pre_n[k] = reinterpret_cast<const uint2*>(blk_n + static_cast<size_t>(j) * kRowVec)[lane];
         }
-        // ------------------------------------------------------------ a4: K rows out, V rows in behind them
+        double folded_next = 0.0;
+        if (next_share && tid < kHeadDim) folded_next = fold_running_sum(un);   // (its loads arrive under the stores)
         {
             uint4* out = p.k_cache + static_cast<size_t>(u) * N * kRowVec;
             if (kOnePass && crank == 0 && un + nclusters < p.U) {   // the block rows of the unit after next towards L2
@@ -1121,9 +1126,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 const bool vis = lr < seg && lr >= skip_local;
                 const int d = vis ? dst_of[lr] : -1;
                 if (d >= 0) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
-                if (vis && d < 0 && use_stash && seg_a + lr < len) {   // an evicted cache row: kept aside as it is
-                    uint4* srow = stash + (evicted_before(seg_a + lr) - eb_lo) * kRowVec;
-                    srow[t] = ra[k]; srow[t + 8] = rb[k];
+                // evicted cache rows among the warp's four: one at a time through the warp's scratch row, re-read one
+                // warp per row
+                for (unsigned gm = __ballot_sync(0xffffffffu, vis && d < 0 && seg_a + lr < len) & 0x01010101u; gm; gm &= gm - 1) {
+                    const int gsub = (__ffs(gm) - 1) >> 3;
+                    __syncwarp();
+                    if (sub == gsub) { warp_row[warp * kRowVec + t] = ra[k]; warp_row[warp * kRowVec + t + 8] = rb[k]; }
+                    __syncwarp();
+                    warp_row_terms(reinterpret_cast<const uint2*>(warp_row + warp * kRowVec)[lane], true, inv_eps, raw, acc_g);
                 }
                 if (vis) {
                     const uint4* row = concat_row(p.v_cache, p.new_v, u, seg_a + lr, len, B, N);
@@ -1141,9 +1151,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                     const bool vis = lr < rs && lr >= skip_local;
                     const int d = vis ? dst_of[lr] : -1;
                     if (d >= 0) { out[d * kRowVec + t] = rows[lr * kRowVec + t]; out[d * kRowVec + t + 8] = rows[lr * kRowVec + t + 8]; }
-                    if (vis && d < 0 && use_stash && seg_a + lr < len) {   // an evicted cache row: kept aside as it is
-                        uint4* srow = stash + (evicted_before(seg_a + lr) - eb_lo) * kRowVec;
-                        srow[t] = rows[lr * kRowVec + t]; srow[t + 8] = rows[lr * kRowVec + t + 8];
+                    // evicted cache rows among these four (rare): their terms, one warp per row, straight from the tile
+                    for (unsigned gm = __ballot_sync(0xffffffffu, vis && d < 0 && seg_a + lr < len) & 0x01010101u; gm; gm &= gm - 1) {
+                        const int glr = tile * kTileRows + it * 4 + ((__ffs(gm) - 1) >> 3);
+                        warp_row_terms(reinterpret_cast<const uint2*>(rows + glr * kRowVec)[lane], true, inv_eps, raw, acc_g);
                     }
                 }
                 // The tile's only readers are this warp's lanes and their reads have returned (the stores
@@ -1154,80 +1165,29 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             }
         }
         KD_STAMP(6);
-        // ------------------------------------------------------------ while the V rows arrive: terms of the rows that left,
-        // and this CTA's share of the next unit's block
-        double folded_next = 0.0, share_next = 0.0;
+        // ------------------------------------------------------------ the block rows of this CTA's range (requested before the
+        // stores), every warp's sums into the tables, one barrier, and the delta and the next share are complete
+        double share_next = 0.0;
         {
-            const bool next_share = kOnePass && un < p.U;
-            if (next_share && tid < kHeadDim) folded_next = fold_running_sum(un);   // (its loads arrive under what follows)
-            __syncthreads();   // the stash is complete
-            const int n_st = use_stash ? n_gone_cache : 0;
-            const uint4* blk_u = p.new_k + static_cast<size_t>(u) * B * kRowVec;
-            const uint4* blk_n = p.new_k + static_cast<size_t>(next_share ? un : u) * B * kRowVec;
-            const int c = tid & (kHeadDim - 1), q = tid >> 7;
-            double gone = 0.0, nxt = 0.0;
-            for (int r0 = b_lo; r0 == b_lo || r0 < b_hi; r0 += kHeadDim) {   // 128 block rows of the range at a time (usually all)
-                const int mc = max(0, min(kHeadDim, b_hi - r0));
-                const int st0 = r0 == b_lo ? n_st : 0;                        // the stash goes with the first chunk
-                const int items = st0 + mc + (next_share ? mc : 0);
-                if (r0 > b_lo) __syncthreads();   // the previous chunk's reciprocal norms have been read
-                // phase 1: one row group per row: 1 / ||k||
-                for (int i0 = 0; i0 + 4 * warp < items; i0 += kGroups) {   // (warp-uniform bound: pairs_sumsq shuffles)
-                    int it = i0 + g;
-                    uint4 a = make_uint4(0, 0, 0, 0), b = a;
-                    float* inv_out = nullptr;
-                    if (it < st0) {
-                        a = stash[it * kRowVec + t]; b = stash[it * kRowVec + t + 8];
-                        inv_out = inv_st + it;
-                    } else if ((it -= st0) < mc) {
-                        const int i = len + r0 + it;   // token index of block row r0 + it
-                        if ((bitmap[i >> 5] >> (i & 31)) & 1u) {
-                            const uint4* row = blk_u + static_cast<size_t>(r0 + it) * kRowVec;
-                            a = row[t]; b = row[t + 8];
-                            inv_out = inv_ev + it;
-                        } else if (t == 0) {
-                            inv_ev[it] = 0.f;   // kept: no term
-                        }
-                    } else if ((it -= mc) < mc && next_share) {
-                        const uint4* row = blk_n + static_cast<size_t>(r0 + it) * kRowVec;
-                        a = row[t]; b = row[t + 8];
-                        inv_out = inv_nx + it;
-                    }
-                    float2 x[8];
-                    unpack_pairs(a, b, x);
-                    const float ss = pairs_sumsq(x);
-                    if (inv_out && t == 0) *inv_out = raw ? 1.0f : fminf(approx_rsqrt(ss), inv_eps);
-                }
-                __syncthreads();
-                // phase 2: thread (channel c, quarter q) adds rows q, q + 4, ... of its channel, in order, in double
-                for (int j = q; j < st0; j += 4) {
-                    const uint32_t h = reinterpret_cast<const uint16_t*>(stash + j * kRowVec)[c];
-                    gone += static_cast<double>(__fmul_rn(__uint_as_float(h << 16), inv_st[j]));
-                }
-                for (int jb = q; jb < mc; jb += 32) {   // eight rows' elements requested before the first is used
-                    uint32_t he[8], hn[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int j = jb + 4 * i;
-                        he[i] = (j < mc && inv_ev[j] != 0.f) ? __ldg(reinterpret_cast<const uint16_t*>(blk_u + static_cast<size_t>(r0 + j) * kRowVec) + c) : 0u;
-                        hn[i] = (j < mc && next_share) ? __ldg(reinterpret_cast<const uint16_t*>(blk_n + static_cast<size_t>(r0 + j) * kRowVec) + c) : 0u;
-                    }
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int j = jb + 4 * i;
-                        if (j < mc && inv_ev[j] != 0.f) gone += static_cast<double>(__fmul_rn(__uint_as_float(he[i] << 16), inv_ev[j]));
-                        if (j < mc && next_share) nxt += static_cast<double>(__fmul_rn(__uint_as_float(hn[i] << 16), inv_nx[j]));
-                    }
-                }
+            for (int k = 0; k < kPreRows; ++k) {
+                const int j = b_lo + warp + k * kFusedWarps;   // (warp-uniform conditions)
+                if (block_row_evicted(j)) warp_row_terms(pre_e[k], true, inv_eps, raw, acc_g);
+                if (next_share && j < b_hi) warp_row_terms(pre_n[k], true, inv_eps, raw, acc_n);
             }
-            part_g[q * kHeadDim + c] = gone;
-            part_n[q * kHeadDim + c] = nxt;
+            for (int j = b_lo + warp + kPreRows * kFusedWarps; j < b_hi; j += kFusedWarps) {   // ranges of more than 32 rows
+                if (block_row_evicted(j))
+                    warp_row_terms(reinterpret_cast<const uint2*>(blk_u + static_cast<size_t>(j) * kRowVec)[lane], true, inv_eps, raw, acc_g);
+                if (next_share)
+                    warp_row_terms(reinterpret_cast<const uint2*>(blk_n + static_cast<size_t>(j) * kRowVec)[lane], true, inv_eps, raw, acc_n);
+            }
+            store_warp_sums(acc_g, gone_tab, warp, lane);
+            store_warp_sums(acc_n, next_tab, warp, lane);
             __syncthreads();
             if (tid < kHeadDim) {
-                const double gsum = gone_rounds + ((part_g[c] + part_g[kHeadDim + c]) + (part_g[2 * kHeadDim + c] + part_g[3 * kHeadDim + c]));
-                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass ? my_share : 0.0) - gsum;
+                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass ? my_share : 0.0) - sum_warp_sums(gone_tab, tid);
                 if (next_share) {
-                    share_next = (part_n[c] + part_n[kHeadDim + c]) + (part_n[2 * kHeadDim + c] + part_n[3 * kHeadDim + c]);
+                    share_next = sum_warp_sums(next_tab, tid);
                     push_share(share_next);   // read by every CTA after the third cluster barrier
                 }
             }
@@ -1272,6 +1232,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                     ra[k] = row[t]; rb[k] = row[t + 8];
                 }
             }
+            // V tiles out, the next unit's K tile in behind each, and -- one-pass steps -- the K tile that went in
+            // behind the PREVIOUS V tile scored while this one's stores drain: the arithmetic runs under the copies
+            const bool score_next = kOnePass && un < p.U;
+            float2 w[8];
+            float m = 0.f;
+            if (score_next) {
+                const float* mu_next = mu_buf + (cur ^ 1) * kHeadDim;
+                load_anchor(mu_next, t, w);
+                m = anchor_norm(mu_next, lane);
+            }
+            int prev = -1;   // this warp's previous tile slot: its K tile of the next unit is not scored yet
 #pragma unroll 1
             for (int s = 0; s < kTilesPerWarp; ++s) {
                 const int tile = warp + kFusedWarps * s;
@@ -1288,28 +1259,24 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                     __syncwarp();
                 }
                 if (lane == 0 && un < p.U) issue_tile(p.k_cache, p.new_k, un, len, B, N, sl, tile, rows_sa, mbar_sa);
+                if (score_next && prev >= 0) {
+                    mbar_wait(mbar_sa + 8 * (warp + kFusedWarps * prev), (parity >> prev) & 1u, p.status);
+                    parity ^= 1u << prev;
+                    score_tile(rows, warp + kFusedWarps * prev, rs, t, sub, w, m, p.eps, keys + seg_a);
+                }
+                prev = s;
+            }
+            if (score_next && prev >= 0) {
+                mbar_wait(mbar_sa + 8 * (warp + kFusedWarps * prev), (parity >> prev) & 1u, p.status);
+                parity ^= 1u << prev;
+                score_tile(rows, warp + kFusedWarps * prev, rs, t, sub, w, m, p.eps, keys + seg_a);
             }
         }
         KD_STAMP(10);
         if (kOnePass && un < p.U) {
-            // the next unit's tiles, scored by their warp as they land behind the V rows (the first ones have had the
-            // time the later ones took to leave); the key table is free: every CTA has passed the third barrier
-            float2 w[8];
-            const float* mu_next = mu_buf + (cur ^ 1) * kHeadDim;
-            load_anchor(mu_next, t, w);
-            const float m = anchor_norm(mu_next, lane);
-#pragma unroll 1
-            for (int s = 0; s < kTilesPerWarp; ++s) {
-                const int tile = warp + kFusedWarps * s;
-                if (tile >= ntiles) break;
-                mbar_wait(mbar_sa + 8 * tile, (parity >> s) & 1u, p.status);
-                parity ^= 1u << s;
-                score_tile(rows, tile, rs, t, sub, w, m, p.eps, keys + seg_a);
-            }
             tiles_scored = true;
             cur ^= 1;
             my_share = share_next;
-            folded = folded_next;
         }
         KD_STAMP(11);
         __syncthreads();   // dst_of is free for the next unit
