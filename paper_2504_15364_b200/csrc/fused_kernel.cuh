@@ -52,7 +52,7 @@ constexpr int kCandCap = kFusedThreads;                 // exact-rank stage hand
 constexpr int kMaxCluster = 16;
 constexpr int kFastKeys = 17;                           // fast select: keys per thread held in registers (n <= 8704)
 constexpr int kFastCandCap = 192;                       // fast select: keys of the threshold bin ranked exactly
-constexpr int kReduceBytes = 32 * 1024;   // scratch the dead key table lends: staged row terms (16 KB), quarter sums, lists
+constexpr int kReduceBytes = 16 * 1024;   // scratch the dead key table lends: staged row terms (16 KB), quarter sums, lists
 constexpr int kSmemLimit = 232448;                      // opt-in shared memory per CTA on sm_100
 constexpr int kErrTimeout = -6;                         // KEYDIFF_ERR_TIMEOUT
 constexpr uint32_t kWaitSpins = 1u << 24;               // bound of every mbarrier wait
@@ -74,7 +74,7 @@ __host__ __device__ inline FusedLayout fused_layout(int smem_rows, int nkeys, in
     L.bitmap = take(2 * ((nkeys + 31) / 32) * 4);   // evicted-token bitmap, evicted-before count of every word
     L.sel = take(static_cast<int>(sizeof(SelectSmem)));
     L.mu = take(2 * kHeadDim * 4);   // this unit's anchor and the next unit's
-    L.mbar = take(kMaxTiles * 8);
+    L.mbar = take((kMaxTiles + 1) * 8);   // one per tile + the key exchange's
     L.misc = take(128);
     L.total = off;
     return L;
@@ -133,6 +133,15 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// this CTA's shared memory -> a peer CTA's shared memory (cluster addresses of the destination and of the PEER's
+// mbarrier, which counts the bytes as they land); 16-byte aligned, size % 16 == 0.  A plain peer-to-peer copy inside
+// the cluster: no multicast.
+__device__ __forceinline__ void bulk_push(uint32_t dst_cluster, uint32_t src, uint32_t bytes, uint32_t bar_cluster) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster), "r"(src), "r"(bytes), "r"(bar_cluster) : "memory");
+}
+// orders this thread's earlier shared-memory writes in front of later reads of them by the copy engine
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t;
 }
@@ -748,20 +757,28 @@ __device__ __forceinline__ void warp_row_terms(uint2 wds, bool active, float inv
         acc[2] += static_cast<double>(__fmul_rn(x2, inv)); acc[3] += static_cast<double>(__fmul_rn(x3, inv));
     }
 }
-// A warp's four sums per lane (channels 4l .. 4l+3) into its row of a [16 warps][128] table of doubles.
-__device__ __forceinline__ void store_warp_sums(const double (&acc)[4], double* table, int warp, int lane) {
-    double2* row = reinterpret_cast<double2*>(table + warp * kHeadDim + 4 * lane);
-    row[0] = make_double2(acc[0], acc[1]);
-    row[1] = make_double2(acc[2], acc[3]);
-}
-// Channel c's total over the 16 warps, in warp order.
-__device__ __forceinline__ double sum_warp_sums(const double* table, int c) {
+// The 16 warps' four sums per lane (channels 4l .. 4l+3) added up over the CTA in a fixed order through an
+// [8][128] table of doubles: warps 0..7 store their sums, warps 8..15 add theirs to the row of warp w - 8, and
+// channel c's total is the sum of the eight rows in order.  Returns the total in threads tid < 128 (0 elsewhere).
+// Two CTA barriers inside; the caller synchronises before the table is reused.
+__device__ __forceinline__ double cta_sum_of_warp_sums(const double (&acc)[4], double* table, int tid) {
+    const int warp = tid >> 5, lane = tid & 31;
+    double2* row = reinterpret_cast<double2*>(table + (warp & 7) * kHeadDim + 4 * lane);
+    if (warp < 8) { row[0] = make_double2(acc[0], acc[1]); row[1] = make_double2(acc[2], acc[3]); }
+    __syncthreads();
+    if (warp >= 8) {
+        const double2 a = row[0], b = row[1];
+        row[0] = make_double2(a.x + acc[0], a.y + acc[1]); row[1] = make_double2(b.x + acc[2], b.y + acc[3]);
+    }
+    __syncthreads();
     double s = 0.0;
+    if (tid < kHeadDim) {
 #pragma unroll
-    for (int w = 0; w < kFusedWarps; ++w) s += table[w * kHeadDim + c];
+        for (int w = 0; w < 8; ++w) s += table[w * kHeadDim + tid];
+    }
     return s;
 }
-constexpr int kPreRows = 2;   // block rows per warp and kind requested before the K stores (the rest after them)
+constexpr int kPreRows = 4;   // block rows per warp and kind requested before the K stores (the rest after them)
 
 // kRegRows = rows per row group that live in registers (the host picks the smallest instance that
 // holds a slice together with the shared-memory rows).
@@ -798,8 +815,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     const uint32_t keys_sa = smem_addr(keys), partials_sa = smem_addr(partials);
     // scratch that the dead key table lends between the selection and the third cluster barrier (no peer writes the
     // table in that window): every warp's sums of the terms that left and of the next block's terms
-    double* gone_tab = reinterpret_cast<double*>(keys);                 // [16][128]
-    double* next_tab = gone_tab + kFusedWarps * kHeadDim;               // [16][128]
+    double* gone_tab = reinterpret_cast<double*>(keys);                 // [8][128]: warps w and w + 8 share row w
+    double* next_tab = gone_tab + (kFusedWarps / 2) * kHeadDim;         // [8][128]
     uint4* warp_row = reinterpret_cast<uint4*>(smem + L.xchg);          // [16 warps][16 words]: a register-resident row, re-read
                                                                         // one warp per row (the candidates' area, dead by then)
 
@@ -818,17 +835,18 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     sl.seg = min(n, sl.seg_a + p.rows_per_cta) - sl.seg_a;
     sl.rs = min(sl.seg, p.smem_rows);
     sl.ntiles = (sl.rs + kTileRows - 1) / kTileRows;
-    const int seg_a = sl.seg_a, seg = sl.seg, seg_b = seg_a + seg, rs = sl.rs, ntiles = sl.ntiles;
+    const int seg_a = sl.seg_a, seg = sl.seg, rs = sl.rs, ntiles = sl.ntiles;
     // Shared-memory rows are handled tile by tile (16 rows); warp w owns tiles w, w+16, w+32, ... in
     // every phase, so a tile is loaded, read, written out and refilled by one warp: the hand-over of
     // a tile from its readers to the copy engine needs a __syncwarp, never a CTA-wide barrier.
 
     if (tid == 0) {
-        for (int j = 0; j < kMaxTiles; ++j) mbar_init(mbar_sa + 8 * j, 1);
+        for (int j = 0; j <= kMaxTiles; ++j) mbar_init(mbar_sa + 8 * j, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     uint32_t parity = 0;   // bit s: phase parity the next wait on this warp's s-th tile expects
+    uint32_t xparity = 0;  // phase parity of the key exchange's barrier
 
     // All clusters start together and do identical work per unit, so left alone they stay in lock
     // step: every SM loads at the same moment, then every SM computes while HBM idles.  Starting
@@ -863,7 +881,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     // [b_lo, b_hi), pushes its share of their sum of terms into every peer's table (DSMEM), and after a cluster
     // barrier every CTA adds the C shares in rank order to the folded running sum: the same anchor bits everywhere.
     const int b_per = (B + C - 1) / C;
-    const int b_lo = min(B, crank * b_per), b_hi = min(B, b_lo + b_per), nb = b_hi - b_lo;
+    const int b_lo = min(B, crank * b_per), b_hi = min(B, b_lo + b_per);
     double my_share = 0.0;       // tid < 128: channel tid of this CTA's share of this unit's block sum
     bool tiles_scored = false;   // this unit's tiles were scored behind the previous unit's V rows
     int cur = 0;                 // which of the two anchor buffers holds this unit's anchor
@@ -895,9 +913,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             const uint4* blk = p.new_k + static_cast<size_t>(cluster_id) * B * kRowVec;
             for (int j = b_lo + warp; j < b_hi; j += kFusedWarps)   // (warp-uniform)
                 warp_row_terms(reinterpret_cast<const uint2*>(blk + static_cast<size_t>(j) * kRowVec)[lane], true, inv_eps, raw, acc);
-            store_warp_sums(acc, gone_tab, warp, lane);   // (nobody uses the key table before the first unit's scores)
-            __syncthreads();
-            if (tid < kHeadDim) my_share = sum_warp_sums(gone_tab, tid);
+            my_share = cta_sum_of_warp_sums(acc, gone_tab, tid);   // (nobody uses the key table before the first unit's scores)
             __syncthreads();   // the table is free again before any key is written
         }
         if (tid < kHeadDim) push_share(my_share);
@@ -1031,17 +1047,29 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             }
         }   // kOnePass
         KD_STAMP(1);
+        // this slice's keys -> every peer's table: one bulk copy per peer, counted on the PEER's exchange barrier; a CTA
+        // goes on as soon as its own table is complete (n - seg keys have landed), no cluster-wide barrier.  The
+        // peers' tables are free: nobody writes a unit's keys before it has passed the previous unit's third barrier.
+        fence_proxy_async_smem();   // this thread's keys, in front of the copy engine's reads
         __syncthreads();
-        {
-            // this slice's keys -> every peer's table (128-bit DSMEM stores)
-            const uint4* mine = reinterpret_cast<const uint4*>(keys + seg_a);
-            for (int c = 1; c < C; ++c) {
-                const int peer = crank + c < C ? crank + c : crank + c - C;
-                const uint32_t base = map_to_cta(keys_sa + 4 * seg_a, peer);
-                for (int o = tid; 4 * o < seg; o += kFusedThreads) st_cluster_v4(base + 16 * o, mine[o]);
+        if (tid == 0) {
+            // (a bulk copy moves multiples of 16 bytes: a ragged last slice is sent with up to three entries of
+            // padding, which land beyond key n - 1 inside the sender's own part of the table and are never read)
+            const uint32_t xbar = mbar_sa + 8 * kMaxTiles;
+            uint32_t expected = 0;
+            for (int c = 0; c < C; ++c) {
+                const int a = min(n, c * p.rows_per_cta), sg = min(n, a + p.rows_per_cta) - a;
+                if (c != crank) expected += static_cast<uint32_t>((sg + 3) & ~3) * 4u;
+            }
+            mbar_expect_tx(xbar, expected);   // what the peers will send here
+            if (seg > 0) {
+                const uint32_t bytes = static_cast<uint32_t>((seg + 3) & ~3) * 4u;
+                for (int c = 1; c < C; ++c) {
+                    const uint32_t peer = static_cast<uint32_t>(crank + c < C ? crank + c : crank + c - C);
+                    bulk_push(map_to_cta(keys_sa + 4 * seg_a, peer), keys_sa + 4 * seg_a, bytes, map_to_cta(xbar, peer));
+                }
             }
         }
-        cluster_arrive();
         {
             float* sc = p.scores + static_cast<size_t>(u) * p.nmax + seg_a;   // fp32 scores to global scratch, coalesced
             for (int lr = tid; lr < seg; lr += kFusedThreads) sc[lr] = key_score(keys[seg_a + lr]);
@@ -1049,7 +1077,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;
             if (tid == 0) { misc[0] = 0; misc[1] = n; }
         }
-        cluster_wait();       // (2) the key table of every CTA holds all n keys
+        mbar_wait(mbar_sa + 8 * kMaxTiles, xparity, p.status);   // (2) this CTA's key table holds all n keys
+        xparity ^= 1u;
+        __syncthreads();   // (the zeroing above is complete as well)
         KD_STAMP(2);
         if (p.window > 0) {
             // sliding window (Sec. 3.2): the last `window` tokens get the largest possible key, so they are
@@ -1126,9 +1156,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 const bool vis = lr < seg && lr >= skip_local;
                 const int d = vis ? dst_of[lr] : -1;
                 if (d >= 0) { out[d * kRowVec + t] = ra[k]; out[d * kRowVec + t + 8] = rb[k]; }
-                // evicted cache rows among the warp's four: one at a time through the warp's scratch row, re-read one
-                // warp per row
-                for (unsigned gm = __ballot_sync(0xffffffffu, vis && d < 0 && seg_a + lr < len) & 0x01010101u; gm; gm &= gm - 1) {
+                // evicted cache rows among the warp's four (a nibble of the bitmap says whether there is any): one at a
+                // time through the warp's scratch row, re-read one warp per row
+                const int i4 = seg_a + rs + k * kGroups + 4 * warp;   // the warp's four rows are tokens i4 .. i4 + 3 (i4 % 4 == 0)
+                const bool any_gone = i4 < len && ((bitmap[i4 >> 5] >> (i4 & 31)) & 0xfu) != 0;   // (warp-uniform)
+                for (unsigned gm = any_gone ? __ballot_sync(0xffffffffu, vis && d < 0 && seg_a + lr < len) & 0x01010101u : 0u; gm; gm &= gm - 1) {
                     const int gsub = (__ffs(gm) - 1) >> 3;
                     __syncwarp();
                     if (sub == gsub) { warp_row[warp * kRowVec + t] = ra[k]; warp_row[warp * kRowVec + t + 8] = rb[k]; }
@@ -1145,6 +1177,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 const int tile = warp + kFusedWarps * s;
                 if (tile >= ntiles) break;
                 if (min(rs, (tile + 1) * kTileRows) <= skip_local) continue;   // no row of the tile moves
+                // the bitmap bits of the tile's 16 tokens (they may straddle two words; a word past the end only adds
+                // bits that the exact test below rejects)
+                const int i16 = seg_a + tile * kTileRows;
+                const unsigned gone16 = i16 < len ? __funnelshift_r(bitmap[i16 >> 5], bitmap[(i16 >> 5) + 1], i16 & 31) & 0xffffu : 0u;   // (warp-uniform)
 #pragma unroll
                 for (int it = 0; it < 4; ++it) {
                     const int lr = tile * kTileRows + it * 4 + sub;
@@ -1152,7 +1188,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                     const int d = vis ? dst_of[lr] : -1;
                     if (d >= 0) { out[d * kRowVec + t] = rows[lr * kRowVec + t]; out[d * kRowVec + t + 8] = rows[lr * kRowVec + t + 8]; }
                     // evicted cache rows among these four (rare): their terms, one warp per row, straight from the tile
-                    for (unsigned gm = __ballot_sync(0xffffffffu, vis && d < 0 && seg_a + lr < len) & 0x01010101u; gm; gm &= gm - 1) {
+                    for (unsigned gm = ((gone16 >> (4 * it)) & 0xfu) ? __ballot_sync(0xffffffffu, vis && d < 0 && seg_a + lr < len) & 0x01010101u : 0u; gm; gm &= gm - 1) {
                         const int glr = tile * kTileRows + it * 4 + ((__ffs(gm) - 1) >> 3);
                         warp_row_terms(reinterpret_cast<const uint2*>(rows + glr * kRowVec)[lane], true, inv_eps, raw, acc_g);
                     }
@@ -1181,13 +1217,30 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 if (next_share)
                     warp_row_terms(reinterpret_cast<const uint2*>(blk_n + static_cast<size_t>(j) * kRowVec)[lane], true, inv_eps, raw, acc_n);
             }
-            store_warp_sums(acc_g, gone_tab, warp, lane);
-            store_warp_sums(acc_n, next_tab, warp, lane);
-            __syncthreads();
+            // (both tables go through their two barriers together)
+            {
+                double2* rg = reinterpret_cast<double2*>(gone_tab + (warp & 7) * kHeadDim + 4 * lane);
+                double2* rn = reinterpret_cast<double2*>(next_tab + (warp & 7) * kHeadDim + 4 * lane);
+                if (warp < 8) {
+                    rg[0] = make_double2(acc_g[0], acc_g[1]); rg[1] = make_double2(acc_g[2], acc_g[3]);
+                    rn[0] = make_double2(acc_n[0], acc_n[1]); rn[1] = make_double2(acc_n[2], acc_n[3]);
+                }
+                __syncthreads();
+                if (warp >= 8) {
+                    double2 a = rg[0], b = rg[1];
+                    rg[0] = make_double2(a.x + acc_g[0], a.y + acc_g[1]); rg[1] = make_double2(b.x + acc_g[2], b.y + acc_g[3]);
+                    a = rn[0]; b = rn[1];
+                    rn[0] = make_double2(a.x + acc_n[0], a.y + acc_n[1]); rn[1] = make_double2(b.x + acc_n[2], b.y + acc_n[3]);
+                }
+                __syncthreads();
+            }
             if (tid < kHeadDim) {
-                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass ? my_share : 0.0) - sum_warp_sums(gone_tab, tid);
+                double gsum = 0.0, nsum = 0.0;
+#pragma unroll
+                for (int w = 0; w < 8; ++w) { gsum += gone_tab[w * kHeadDim + tid]; nsum += next_tab[w * kHeadDim + tid]; }
+                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass ? my_share : 0.0) - gsum;
                 if (next_share) {
-                    share_next = sum_warp_sums(next_tab, tid);
+                    share_next = nsum;
                     push_share(share_next);   // read by every CTA after the third cluster barrier
                 }
             }

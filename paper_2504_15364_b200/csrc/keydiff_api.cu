@@ -171,7 +171,7 @@ int max_active_clusters(Kernel kern, int C, int smem, int sm_count) {
 // picks the winner (constants from per-phase timings of the kernel on a B200).
 bool plan_fused(keydiff_ctx* c, int sm_count) {
     using namespace kd;
-    constexpr double kUnitFixedUs = 10.3, kRowUs = 0.0202;
+    constexpr double kUnitFixedUs = 10.0, kRowUs = 0.0165, kManyRegRowsUs = 4.5;   // (more than 4 register rows: spills)
     const int forced = c->tune_cluster;
     double best = 0.0;
     bool found = false;
@@ -189,7 +189,8 @@ bool plan_fused(keydiff_ctx* c, int sm_count) {
         const int clusters = max_active_clusters(kern, C, smem, sm_count);
         if (clusters < 1) continue;
         const int used = std::min(c->U, clusters);
-        const double est = static_cast<double>((c->U + used - 1) / used) * (kUnitFixedUs + kRowUs * per_cta);
+        const double est = static_cast<double>((c->U + used - 1) / used) *
+                           (kUnitFixedUs + kRowUs * per_cta + (reg_rows > 4 ? kManyRegRowsUs : 0.0));
         if (!found || est < 0.95 * best) {   // a larger cluster has to pay for its extra barrier traffic
             found = true; best = est;
             c->cluster = C; c->fused_smem_rows = sr; c->fused_nkeys = nkeys; c->fused_smem_bytes = smem;
