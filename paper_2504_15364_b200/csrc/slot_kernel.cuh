@@ -83,18 +83,6 @@ __device__ __forceinline__ void issue_rows(const uint4* cache, const uint4* bloc
                   block + (static_cast<size_t>(u) * B + (g0 + from_cache - len)) * kRowVec, from_block * kRowBytes, bar);
 }
 
-// Row j of a CTA's share of a list of candidate numbers: entry (j / 64) * step + base + j % 64 of the list (the
-// share is every `step / 64`-th run of 64 entries), as a pointer to that candidate's key row.  A list entry
-// outside [0, n) cannot occur; the clamp makes sure that even then no address outside the tensors is formed.
-struct ListedRows {
-    const uint4* cache; const uint4* block; const int* list;
-    int u, len, B, N, n, step, base;
-    __device__ __forceinline__ const uint4* operator()(int j) const {
-        const int v = list[(j / kGroups) * step + base + (j % kGroups)];
-        return concat_row(cache, block, u, min(max(v, 0), n - 1), len, B, N);
-    }
-};
-
 __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const SlotParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int C = p.cluster;
@@ -178,13 +166,24 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
                 for (int c = 0; c < kMaxCluster; ++c)
                     dl[c] = c < C ? p.anchor_delta[(static_cast<size_t>(u) * C + c) * kHeadDim + tid] : 0.0;
             }
-            // every CTA normalises the whole block itself; scratch: the work area (the key table cannot lend its space
-            // here: a peer that is ahead may already be pushing its keys of this unit into it)
+            // every CTA normalises the whole block itself, one warp per row (the canonical form of a row's terms, see
+            // fused_kernel.cuh), eight rows requested at a time; scratch: the work area (the key table cannot lend its
+            // space here: a peer that is ahead may already be pushing its keys of this unit into it)
             {
-                const ContiguousRows blk{p.new_k + static_cast<size_t>(u) * B * kRowVec};
-                block_sum = global_rows_terms_sum(blk, B, inv_eps, raw,
-                                                  reinterpret_cast<float*>(smem + L.work) + 8 * kHeadDim,
-                                                  reinterpret_cast<double*>(smem + L.work), tid);
+                const uint4* blk = p.new_k + static_cast<size_t>(u) * B * kRowVec;
+                double acc[4] = {0.0, 0.0, 0.0, 0.0};
+                for (int j0 = warp; j0 < B; j0 += 8 * kFusedWarps) {   // (warp-uniform)
+                    uint2 wds[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int j = j0 + k * kFusedWarps;
+                        wds[k] = j < B ? reinterpret_cast<const uint2*>(blk + static_cast<size_t>(j) * kRowVec)[lane] : make_uint2(0, 0);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (j0 + k * kFusedWarps < B) warp_row_terms(wds[k], true, inv_eps, raw, acc);
+                }
+                block_sum = cta_sum_of_warp_sums(acc, reinterpret_cast<double*>(smem + L.work), tid);
             }
             if (tid < kHeadDim) {
                 double a = run;
@@ -342,17 +341,31 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
             // (a) evicted rows, read once more (from L2): their terms leave the running sum.  The CTA that re-reads
             // evicted row r is the one that overwrites its slot in (b): rows r with (r / 64) % C == crank.
             const int stride = C * kGroups, r_first = crank * kGroups + g;
-            double gone = 0.0;   // tid < 128: channel tid of this CTA's evicted rows' sum of terms
             {
                 const int rem = E % stride - crank * kGroups;
                 const int mine = (E / stride) * kGroups + min(max(rem, 0), kGroups);
-                const uint4* kc = p.k_cache; const uint4* nk = p.new_k;
-                float* inv_sh = reinterpret_cast<float*>(keys);   // the key table is dead until the next unit
-                const ListedRows rows_of{kc, nk, ev_of, u, len, B, N, n, stride, crank * kGroups};
-                gone = global_rows_terms_sum(rows_of, mine, inv_eps, raw, inv_sh, reinterpret_cast<double*>(inv_sh + kHeadDim), tid);
+                double acc[4] = {0.0, 0.0, 0.0, 0.0};
+                for (int j0 = warp; j0 < mine; j0 += 8 * kFusedWarps) {   // one warp per row, eight rows requested at a time
+                    uint2 wds[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int j = j0 + k * kFusedWarps;
+                        wds[k] = make_uint2(0, 0);
+                        if (j < mine) {
+                            const int v = ev_of[(j / kGroups) * stride + crank * kGroups + (j % kGroups)];
+                            // (an entry outside [0, n) cannot occur; the clamp makes sure that even then no address
+                            // outside the tensors is formed)
+                            wds[k] = reinterpret_cast<const uint2*>(concat_row(p.k_cache, p.new_k, u, min(max(v, 0), n - 1), len, B, N))[lane];
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (j0 + k * kFusedWarps < mine) warp_row_terms(wds[k], true, inv_eps, raw, acc);
+                }
+                const double gone = cta_sum_of_warp_sums(acc, reinterpret_cast<double*>(keys), tid);   // the key table is dead until the next unit
                 if (tid < kHeadDim)
                     p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (crank == 0 ? block_sum : 0.0) - gone;
-                __syncthreads();   // every evicted row of this CTA's share has been read: its slot may be overwritten
+                // (the barriers inside the sum lie behind every read of an evicted row: its slot may be overwritten)
             }
             // (b) kept block row r into freed slot r.  For r < evicted_cache that slot is evicted row r, which this
             // same CTA re-read in (a), in front of the barrier above.
