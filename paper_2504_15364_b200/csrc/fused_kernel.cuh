@@ -397,7 +397,7 @@ __device__ __forceinline__ int find_crossing(const int* h, int E, int lane, int 
 }
 
 // Selection at the low end of the key table (every thread of the CTA calls; the result is uniform).  Only
-// E = n - N keys go, so thread t keeps the keys of tokens t, t + 512, ... in registers (n <= 8704); the 2048
+// E = n - N keys go, so thread t looks at the keys of tokens t, t + 512, ... only (in registers up to n = 8704); the 2048
 // bins are spread over the low end of the unit's own key range, from the smallest key to a bound on the
 // E-th smallest (monotone in the key, which is all selection needs); the tokens under the threshold bin go
 // straight into the bitmap, the bin's own few keys are ranked exactly under (key ascending, index
@@ -406,19 +406,29 @@ __device__ __forceinline__ int find_crossing(const int* h, int E, int lane, int 
 // evicted token (both visible to the CTA), or false when the threshold bin holds more than kFastCandCap
 // keys (many equal scores): the bitmap and misc are then in an unspecified state and the caller takes the
 // full-table route.  cand_key / cand_idx: kFastCandCap entries each.
-__device__ __forceinline__ bool low_end_select(const uint32_t* keys, int n, int E, int* hist, uint32_t* bitmap,
-                                               uint32_t* cand_key, int* cand_idx, SelectSmem& sel, int* misc) {
+// kInRegs: the thread's keys stay in registers between the passes (n <= 8704); otherwise they are read again from
+// the table in every pass (any n).
+template <bool kInRegs>
+__device__ __forceinline__ bool low_end_select_impl(const uint32_t* keys, int n, int E, int* hist, uint32_t* bitmap,
+                                                    uint32_t* cand_key, int* cand_idx, SelectSmem& sel, int* misc) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     uint32_t* wmin = reinterpret_cast<uint32_t*>(sel.hist);          // (sel.hist is radix-select scratch)
     uint32_t* wmax = reinterpret_cast<uint32_t*>(sel.hist) + kFusedWarps;
-    const int cnt = (n - tid + kFusedThreads - 1) / kFusedThreads;
-    uint32_t kk[kFastKeys];
+    const int cnt = (n - tid + kFusedThreads - 1) / kFusedThreads;   // keys of this thread: tokens tid, tid + 512, ...
+    constexpr int kSlots = kInRegs ? kFastKeys : 1;
+    uint32_t kk[kSlots];
+    if constexpr (kInRegs) {
 #pragma unroll
-    for (int j = 0; j < kFastKeys; ++j) kk[j] = j < cnt ? keys[tid + j * kFusedThreads] : 0xffffffffu;
+        for (int j = 0; j < kFastKeys; ++j) kk[j] = j < cnt ? keys[tid + j * kFusedThreads] : 0xffffffffu;
+    }
     {
         uint32_t lo = 0xffffffffu, hi = 0u;
+        if constexpr (kInRegs) {
 #pragma unroll
-        for (int j = 0; j < kFastKeys; ++j) { lo = min(lo, kk[j]); if (j < cnt) hi = max(hi, kk[j]); }
+            for (int j = 0; j < kFastKeys; ++j) { lo = min(lo, kk[j]); if (j < cnt) hi = max(hi, kk[j]); }
+        } else {
+            for (int j = 0; j < cnt; ++j) { const uint32_t k = keys[tid + j * kFusedThreads]; lo = min(lo, k); hi = max(hi, k); }
+        }
         // The E-th smallest key is at most the largest of any E distinct keys.  When at least E
         // threads hold keys, the thread minima are such keys, so the largest thread minimum bounds
         // it; otherwise the largest key does.  Keys above the bound share the top bin.
@@ -438,35 +448,51 @@ __device__ __forceinline__ bool low_end_select(const uint32_t* keys, int n, int 
     }
     // bin of a key: linear in the key over [kmin, kcut] (bins 0..2046), 2047 above; monotone
     auto bin_of = [kmin, kcut, shift](uint32_t k) { return k <= kcut ? min((k - kmin) >> shift, 2046u) : 2047u; };
+    // (the top bin holds every key above the bound: the crossing is never there, so it is not counted)
+    if constexpr (kInRegs) {
 #pragma unroll
-    for (int j = 0; j < kFastKeys; ++j) {
-        // (the top bin holds every key above the bound: the crossing is never there, so it is not counted)
-        const uint32_t b = bin_of(kk[j]);
-        if (j < cnt && b != 2047u) atomicAdd(&hist[b], 1);
+        for (int j = 0; j < kFastKeys; ++j) {
+            const uint32_t b = bin_of(kk[j]);
+            if (j < cnt && b != 2047u) atomicAdd(&hist[b], 1);
+        }
+    } else {
+        for (int j = 0; j < cnt; ++j) {
+            const uint32_t b = bin_of(keys[tid + j * kFusedThreads]);
+            if (b != 2047u) atomicAdd(&hist[b], 1);
+        }
     }
     __syncthreads();
     const int packed = find_crossing(hist, E, lane, warp, sel.warp_eq);
     const uint32_t bstar = static_cast<uint32_t>(packed >> 16);
     const int need = E - (packed & 0xffff);   // this many keys of the threshold bin go
-    unsigned m_below = 0, m_in = 0;           // bit j: this thread's j-th key is below / inside the bin
-#pragma unroll
-    for (int j = 0; j < kFastKeys; ++j) {
-        const uint32_t b = bin_of(kk[j]);
-        m_below |= (j < cnt && b < bstar) ? 1u << j : 0u;
-        m_in |= (j < cnt && b == bstar) ? 1u << j : 0u;
-    }
     {
         int first = n;
-        if (packed >= 0 && (m_below | m_in)) {
-            for (unsigned m = m_below; m; m &= m - 1) {
-                const int i = tid + (__ffs(m) - 1) * kFusedThreads;
-                atomicOr(&bitmap[i >> 5], 1u << (i & 31));
-                first = min(first, i);
+        auto evict = [&](int i) { atomicOr(&bitmap[i >> 5], 1u << (i & 31)); first = min(first, i); };
+        auto candidate = [&](uint32_t k, int i) {
+            const int slot = atomicAdd(&misc[0], 1);
+            if (slot < kFastCandCap) { cand_key[slot] = k; cand_idx[slot] = i; }
+        };
+        if constexpr (kInRegs) {
+            unsigned m_below = 0, m_in = 0;           // bit j: this thread's j-th key is below / inside the bin
+#pragma unroll
+            for (int j = 0; j < kFastKeys; ++j) {
+                const uint32_t b = bin_of(kk[j]);
+                m_below |= (j < cnt && b < bstar) ? 1u << j : 0u;
+                m_in |= (j < cnt && b == bstar) ? 1u << j : 0u;
             }
-            for (unsigned m = m_in; m; m &= m - 1) {
-                const int i = tid + (__ffs(m) - 1) * kFusedThreads;
-                const int slot = atomicAdd(&misc[0], 1);
-                if (slot < kFastCandCap) { cand_key[slot] = keys[i]; cand_idx[slot] = i; }
+            if (packed >= 0 && (m_below | m_in)) {
+                for (unsigned m = m_below; m; m &= m - 1) evict(tid + (__ffs(m) - 1) * kFusedThreads);
+                for (unsigned m = m_in; m; m &= m - 1) {
+                    const int i = tid + (__ffs(m) - 1) * kFusedThreads;
+                    candidate(keys[i], i);
+                }
+            }
+        } else if (packed >= 0) {
+            for (int j = 0; j < cnt; ++j) {
+                const int i = tid + j * kFusedThreads;
+                const uint32_t k = keys[i], b = bin_of(k);
+                if (b < bstar) evict(i);
+                else if (b == bstar) candidate(k, i);
             }
         }
         first = __reduce_min_sync(0xffffffffu, first);   // one shared-memory atomic per warp, not per thread
@@ -493,6 +519,15 @@ __device__ __forceinline__ bool low_end_select(const uint32_t* keys, int n, int 
     // Every thread has read misc[0] by now; whoever runs next (the full-table route resets misc) may write it.
     __syncthreads();
     return ok;
+}
+__device__ __noinline__ bool low_end_select_large(const uint32_t* keys, int n, int E, int* hist, uint32_t* bitmap,
+                                                  uint32_t* cand_key, int* cand_idx, SelectSmem& sel, int* misc) {
+    return low_end_select_impl<false>(keys, n, E, hist, bitmap, cand_key, cand_idx, sel, misc);   // (kept out of line: rare)
+}
+__device__ __forceinline__ bool low_end_select(const uint32_t* keys, int n, int E, int* hist, uint32_t* bitmap,
+                                               uint32_t* cand_key, int* cand_idx, SelectSmem& sel, int* misc) {
+    return n <= kFastKeys * kFusedThreads ? low_end_select_impl<true>(keys, n, E, hist, bitmap, cand_key, cand_idx, sel, misc)
+                                          : low_end_select_large(keys, n, E, hist, bitmap, cand_key, cand_idx, sel, misc);
 }
 
 // Exact top-N over the whole key table by one CTA (every CTA of the cluster runs it on its own
@@ -829,7 +864,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     const int nwords = (n + 31) >> 5;
     uint32_t* bitmap = reinterpret_cast<uint32_t*>(smem + L.bitmap);
     int* wlocal = reinterpret_cast<int*>(smem + L.bitmap) + ((p.nkeys + 31) >> 5);
-    const bool fast_ok = n <= kFastKeys * kFusedThreads;   // uniform over the grid
     Slice sl;
     sl.seg_a = min(n, crank * p.rows_per_cta);
     sl.seg = min(n, sl.seg_a + p.rows_per_cta) - sl.seg_a;
@@ -1093,7 +1127,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             // the evicted tokens' bits: selection at the low end of the table, or (crowded threshold bin, large
             // unit) the full-table route; then prefix counts over the bitmap give every kept row of the slice
             // its destination
-            const bool planned = fast_ok && low_end_select(keys, n, E, hist, bitmap, cand_key, cand_idx, sel, misc);
+            const bool planned = low_end_select(keys, n, E, hist, bitmap, cand_key, cand_idx, sel, misc);
             if (!planned) {
                 for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;   // (the attempt may have marked some)
                 __syncthreads();

@@ -109,7 +109,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
     const float inv_eps = 1.0f / p.eps;
     const bool raw = p.raw_anchor != 0;
     const int nwords = (n + 31) >> 5;
-    const bool fast_ok = n <= kFastKeys * kFusedThreads && nwords <= kFusedThreads;
     const int seg_a = min(n, crank * p.rows_per_cta);
     const int seg = min(n, seg_a + p.rows_per_cta) - seg_a, seg_b = seg_a + seg;
     // The slice as a stream of 16-row tiles; warp w takes tiles w, w+16, ... of every unit of the cluster,
@@ -267,7 +266,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
         // ------------------------------------------------------------ a3: the bitmap of evicted candidates
         // the low-end select of fused_kernel.cuh; ties: (key ascending, candidate number descending) go first
         int* wbase = sel.hist + 2 * kFusedWarps;
-        const bool planned = fast_ok && low_end_select(keys, n, E, hist, bitmap, cand_key, cand_idx, sel, misc);
+        const bool planned = low_end_select(keys, n, E, hist, bitmap, cand_key, cand_idx, sel, misc);
         if (!planned) {
             // the full-table select writes the same bitmap (cleared first: the attempt above may have marked some)
             for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;
