@@ -724,6 +724,25 @@ __device__ __forceinline__ double global_rows_terms_sum(RowOf row_of, int count,
 __device__ __forceinline__ void bitmap_prefix(const uint32_t* bitmap, int nwords, int* wlocal, SelectSmem& sel, int* misc) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int* wbase = sel.hist + 2 * kFusedWarps;
+    if (nwords <= kFusedThreads) {   // one word per thread: every warp scans the 16 warp totals itself
+        const int pc = tid < nwords ? __popc(bitmap[tid]) : 0;
+        int incl = pc;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) sel.warp_gt[warp] = incl;
+        __syncthreads();
+        const int t2 = lane < kFusedWarps ? sel.warp_gt[lane] : 0;
+        int incl2 = t2;
+#pragma unroll
+        for (int o = 1; o < 16; o <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl2, o); if (lane >= o) incl2 += v; }
+        const int base = __shfl_sync(0xffffffffu, incl2 - t2, warp);   // evicted tokens before this warp's 32 words
+        if (tid < nwords) wlocal[tid] = base + incl - pc;
+        __syncthreads();
+        return;
+    }
     for (int w0 = 0; w0 < nwords; w0 += kFusedThreads) {
         const int wi = w0 + tid;
         const int pc = wi < nwords ? __popc(bitmap[wi]) : 0;
@@ -956,16 +975,33 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         __syncthreads();
     }
 
+    // one-pass scoring of the register-resident rows (they hold the K rows of the unit to be scored), four at a time
+    auto score_reg_rows = [&](const float2 (&w)[8], float m) {
+#pragma unroll
+        for (int k0 = 0; k0 < kRegRows; k0 += 4) {
+            float vs[4];
+            double vd[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (k0 + i < kRegRows) lane_sumsq_dot(ra[k0 + i], rb[k0 + i], w, vs[i], vd[i]);
+                else { vs[i] = 0.f; vd[i] = 0.0; }
+            }
+            const uint32_t key = score4(vs, vd, t, m, p.eps);
+            const int lr = rs + (k0 + (t >> 1)) * kGroups + g;
+            if (!(t & 1) && k0 + (t >> 1) < kRegRows && lr < seg) keys[seg_a + lr] = key;
+        }
+    };
     KD_STAMP(0);
     for (int u = cluster_id; u < p.U; u += nclusters) {
         const int un = u + nclusters;   // the unit this cluster serves next
         float* mu_sh = mu_buf + cur * kHeadDim;
         if constexpr (kOnePass) {
             // ------------------------------------------------------------ a1 + a2 in one pass: keys of this slice
-            float2 w[8];
-            load_anchor(mu_sh, t, w);
-            const float m = anchor_norm(mu_sh, lane);
+            // (every unit but the cluster's first was scored behind the previous unit's V rows)
             if (!tiles_scored) {
+                float2 w[8];
+                load_anchor(mu_sh, t, w);
+                const float m = anchor_norm(mu_sh, lane);
 #pragma unroll 1
                 for (int s = 0; s < kTilesPerWarp; ++s) {
                     const int tile = warp + kFusedWarps * s;
@@ -974,19 +1010,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                     parity ^= 1u << s;
                     score_tile(rows, tile, rs, t, sub, w, m, p.eps, keys + seg_a);
                 }
-            }
-#pragma unroll
-            for (int k0 = 0; k0 < kRegRows; k0 += 4) {   // register rows, four at a time
-                float vs[4];
-                double vd[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    if (k0 + i < kRegRows) lane_sumsq_dot(ra[k0 + i], rb[k0 + i], w, vs[i], vd[i]);
-                    else { vs[i] = 0.f; vd[i] = 0.0; }
-                }
-                const uint32_t key = score4(vs, vd, t, m, p.eps);
-                const int lr = rs + (k0 + (t >> 1)) * kGroups + g;
-                if (!(t & 1) && k0 + (t >> 1) < kRegRows && lr < seg) keys[seg_a + lr] = key;
+                score_reg_rows(w, m);
             }
         } else {
             // ------------------------------------------------------------ a1: norms and anchor partial
@@ -1149,7 +1173,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             p.first_evicted[u] = first_evicted;
             atomicAdd(p.moved_rows, static_cast<unsigned long long>(N - first_moved));
         }
-        for (int lr = tid; lr < seg; lr += kFusedThreads) {
+        for (int lr = tid; lr < seg; lr += kFusedThreads) {   // kept-index list, coalesced (destinations ascend with lr)
             const int d = dst_of[lr];
             if (d >= 0) {
                 p.kept_idx[static_cast<size_t>(u) * N + d] = seg_a + lr;
@@ -1353,6 +1377,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 }
                 prev = s;
             }
+            if (score_next) score_reg_rows(w, m);   // (their K rows were requested before the tiles: they are here by now)
             if (score_next && prev >= 0) {
                 mbar_wait(mbar_sa + 8 * (warp + kFusedWarps * prev), (parity >> prev) & 1u, p.status);
                 parity ^= 1u << prev;
