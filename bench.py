@@ -244,6 +244,8 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     wl = synth.WORKLOADS[args.workload]
+    if args.batch > 0:
+        wl = synth.scaled(wl, batch=args.batch)
     U, N, B, d = wl.units, wl.budget, wl.block, wl.head_dim
     path = {"auto": binding.KEYDIFF_PATH_AUTO, "staged": binding.KEYDIFF_PATH_STAGED,
             "fused": binding.KEYDIFF_PATH_FUSED}[args.path]
@@ -390,6 +392,9 @@ def main():
     ap.add_argument("--headline-only", action="store_true",
                     help="skip the short runs of the other workloads and of the other layout (the other_workloads list)")
     ap.add_argument("--other-steps", type=int, default=20, help="timed steps of each entry of other_workloads")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="run the workload at this batch size instead of its own (profiling aid: the decode workload's unit shape "
+                         "at batch 2 is 2 GB instead of 34 GB); the line's config says so")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

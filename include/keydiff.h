@@ -23,9 +23,10 @@
  *     time.  Distinct ctxs are independent.
  *   - There is no CPU fallback: on a machine without a usable sm_100 device
  *     keydiff_create fails with KEYDIFF_ERR_CUDA / KEYDIFF_ERR_UNSUPPORTED.
- *   - The environment is read once, by keydiff_create, for three launch-tuning aids (integers; unset =
- *     automatic): KEYDIFF_CLUSTER_SIZE (CTAs per cluster of the fused kernels, 1..16), KEYDIFF_STAGGER_NS
- *     and KEYDIFF_LATE_NS (start-up delays between clusters, nanoseconds).  They change launch shapes
+ *   - The environment is read once, by keydiff_create, for four launch-tuning aids (integers; unset =
+ *     automatic): KEYDIFF_CLUSTER_SIZE (CTAs per cluster of the fused kernels, 1..16), KEYDIFF_MAX_CLUSTERS
+ *     (upper limit on the clusters the ordered fused kernel launches), KEYDIFF_STAGGER_NS and
+ *     KEYDIFF_LATE_NS (start-up delays between clusters, nanoseconds).  They change launch shapes
  *     only, never results; no other call looks at the environment.
  *   - Accuracy of the scores (fp32 storage, fp64 oracle): a score is (mu.k)/(||mu|| ||k||).  The
  *     dot product is accumulated in double precision above chains of four fp32 products, so its error
@@ -66,7 +67,9 @@ enum {
     KEYDIFF_ERR_CUDA = -4,        /* a CUDA runtime call failed; see keydiff_last_cuda_error */
     KEYDIFF_ERR_STATE = -5,       /* call not valid in the ctx's current state */
     KEYDIFF_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired (reported in the status word) */
-    KEYDIFF_ERR_TOO_LARGE = -7    /* keydiff_evict_static: the request does not fit the built-in scratch */
+    KEYDIFF_ERR_TOO_LARGE = -7,   /* keydiff_evict_static: the request does not fit the built-in scratch */
+    KEYDIFF_ERR_INTERNAL = -8     /* status word only, debug-checks build only: a kernel computed a row index outside
+                                     its tensor; the store was skipped */
 };
 
 enum { KEYDIFF_BF16 = 0 };

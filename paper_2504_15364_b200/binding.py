@@ -18,6 +18,7 @@ KEYDIFF_OK = 0
 KEYDIFF_ERR_INVALID_ARG, KEYDIFF_ERR_UNSUPPORTED, KEYDIFF_ERR_ALLOC = -1, -2, -3
 KEYDIFF_ERR_CUDA, KEYDIFF_ERR_STATE, KEYDIFF_ERR_TIMEOUT = -4, -5, -6
 KEYDIFF_ERR_TOO_LARGE = -7
+KEYDIFF_ERR_INTERNAL = -8
 KEYDIFF_BF16 = 0
 KEYDIFF_PATH_AUTO, KEYDIFF_PATH_STAGED, KEYDIFF_PATH_FUSED = 0, 1, 2
 KEYDIFF_ANCHOR_NORMALISED, KEYDIFF_ANCHOR_RAW_MEAN = 0, 1

@@ -23,17 +23,20 @@ def _stale() -> bool:
 
 
 STAMPS_LIB = PKG / "libkeydiff_stamps.so"   # diagnostic build: fused kernel with per-phase timers (phase_times.py)
+DEBUG_LIB = PKG / "libkeydiff_debug.so"     # debug build: computed row indices are range-checked into the status word
 
 
-def build_library(force: bool = False, verbose: bool = False, phase_stamps: bool = False) -> Path:
+def build_library(force: bool = False, verbose: bool = False, phase_stamps: bool = False, debug_checks: bool = False) -> Path:
     """Compile libkeydiff.so in-tree if missing or older than its sources.  phase_stamps=True builds the
-    diagnostic variant libkeydiff_stamps.so instead (-DKEYDIFF_PHASE_STAMPS: the fused kernel times its phases)."""
-    out = STAMPS_LIB if phase_stamps else LIB
-    if not force and not phase_stamps and not _stale():
+    diagnostic variant libkeydiff_stamps.so instead (-DKEYDIFF_PHASE_STAMPS: the fused kernel times its phases),
+    debug_checks=True the variant libkeydiff_debug.so (-DKEYDIFF_DEBUG_CHECKS: row indices are range-checked)."""
+    out = STAMPS_LIB if phase_stamps else DEBUG_LIB if debug_checks else LIB
+    if not force and not phase_stamps and not debug_checks and not _stale():
         return out
     nvcc = os.environ.get("NVCC", "nvcc")
     tmp = out.with_suffix(f".{os.getpid()}.tmp")
-    cmd = [nvcc, *NVCC_FLAGS, *(["-DKEYDIFF_PHASE_STAMPS"] if phase_stamps else []), *(["-Xptxas", "-v"] if verbose else []),
+    cmd = [nvcc, *NVCC_FLAGS, *(["-DKEYDIFF_PHASE_STAMPS"] if phase_stamps else []),
+           *(["-DKEYDIFF_DEBUG_CHECKS"] if debug_checks else []), *(["-Xptxas", "-v"] if verbose else []),
            *map(str, SOURCES), "-o", str(tmp)]
     subprocess.run(cmd, check=True)
     os.replace(tmp, out)
@@ -41,4 +44,5 @@ def build_library(force: bool = False, verbose: bool = False, phase_stamps: bool
 
 
 if __name__ == "__main__":
-    print(build_library(force=True, verbose="-v" in sys.argv, phase_stamps="--phase-stamps" in sys.argv))
+    print(build_library(force=True, verbose="-v" in sys.argv, phase_stamps="--phase-stamps" in sys.argv,
+                        debug_checks="--debug-checks" in sys.argv))

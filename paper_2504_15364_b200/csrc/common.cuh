@@ -10,6 +10,16 @@ constexpr int kRowBytes = kHeadDim * 2;    // bf16 row = 256 B
 constexpr int kRowVec = kRowBytes / 16;    // 16 x 128-bit words per row
 constexpr int kLanesPerRow = 8;            // a row is handled by 8 consecutive lanes
 
+// Debug build (-DKEYDIFF_DEBUG_CHECKS, see build.py --debug-checks): every destination row index a kernel computes
+// is range-checked before the store; a bad index is recorded in the status word (KEYDIFF_ERR_INTERNAL) and the
+// store is skipped.  Without the macro the check is not compiled.
+constexpr int kErrInternal = -8;   // KEYDIFF_ERR_INTERNAL
+#ifdef KEYDIFF_DEBUG_CHECKS
+#define KD_ROW_OK(d, limit, status) ((static_cast<unsigned>(d) < static_cast<unsigned>(limit)) || (atomicExch((status), kd::kErrInternal), false))
+#else
+#define KD_ROW_OK(d, limit, status) true
+#endif
+
 // bf16 is the upper half of a binary32: widening is a shift / a mask.
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }

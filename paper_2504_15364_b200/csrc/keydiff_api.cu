@@ -63,7 +63,7 @@ struct keydiff_ctx {
     int slot_ring_tiles = 0;    //   fused_smem_bytes, fused_max_clusters describe it)
     int slot_nwords = 0;
     int sm_count = 0;           // SMs of the ctx's device
-    int tune_cluster = -1, tune_stagger_ns = -1, tune_late_ns = -1;   // KEYDIFF_* tuning aids as keydiff_create read them
+    int tune_cluster = -1, tune_stagger_ns = -1, tune_late_ns = -1, tune_max_clusters = -1;   // KEYDIFF_* tuning aids as keydiff_create read them
     // running anchor of the fused path: sum of k/||k|| over the cached rows, per unit
     bool incremental = true;    // use it (one-pass kernel) when it is valid
     bool anchor_valid = false;  // the buffers describe the cache as the last evicting step left it
@@ -328,7 +328,8 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     p.raw_anchor = c->cfg.anchor_mode == KEYDIFF_ANCHOR_RAW_MEAN;
     p.window = c->cfg.recent_window;
     p.kept_mirror = c->kept_mirror;
-    const int nclusters = std::min(c->U, c->fused_max_clusters);
+    int nclusters = std::min(c->U, c->fused_max_clusters);
+    if (c->tune_max_clusters > 0) nclusters = std::min(nclusters, c->tune_max_clusters);
     // Start-up stagger: somewhat less than one unit's duration spread evenly over the co-resident
     // clusters.  A unit moves 4 slices (K in, K out, V in, V out) per SM at roughly 60 GB/s per SM when
     // the other SMs are busy too, plus a few microseconds of arithmetic and barriers (a sweep of the
@@ -372,7 +373,7 @@ int launch_staged(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const u
         slot_place_kernel<<<U, kCompactThreads, static_cast<size_t>(B) * 8, st>>>(kc, vc, nk, nv, c->len, B, N, c->kept_idx, c->pos,
                                                                                   static_cast<int>(c->next_pos), c->moved_rows);
     else
-        compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, c->len, B, N, c->kept_idx, c->first_evicted);
+        compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, c->len, B, N, c->kept_idx, c->first_evicted, c->status);
     KD_CUDA(cudaGetLastError());
     return KEYDIFF_OK;
 }
@@ -418,6 +419,7 @@ int create_impl(const keydiff_config* cfg, keydiff_ctx** out) {
     c->tune_cluster = env_int("KEYDIFF_CLUSTER_SIZE");
     c->tune_stagger_ns = env_int("KEYDIFF_STAGGER_NS");
     c->tune_late_ns = env_int("KEYDIFF_LATE_NS");
+    c->tune_max_clusters = env_int("KEYDIFF_MAX_CLUSTERS");
     c->path = KEYDIFF_PATH_STAGED;
     // enough CTAs to fill 148 SMs a few times over, but at least 64 rows per slice
     const int want = (4 * prop.multiProcessorCount + c->U - 1) / c->U;
@@ -704,6 +706,7 @@ const char* keydiff_strerror(int code) {
         case KEYDIFF_ERR_STATE: return "call not valid in the current state (is the ctx's device current?)";
         case KEYDIFF_ERR_TIMEOUT: return "bounded device-side wait expired";
         case KEYDIFF_ERR_TOO_LARGE: return "request needs more scratch than the built-in static scratch array holds";
+        case KEYDIFF_ERR_INTERNAL: return "a kernel computed a row index outside its tensor (debug-checks build)";
         default: return "unknown keydiff status";
     }
 }
@@ -851,7 +854,7 @@ extern "C" int keydiff_evict_static(void* k_cache, void* v_cache, const void* ne
     anchor_partial_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, len, block_B, N, e, rows_per_split, nn, partial, norms, 0);
     score_kernel<<<grid, kStagedThreads, 0, st>>>(kc, nk, len, block_B, N, e, rows_per_split, nn, partial, norms, scores);
     select_kernel<<<U, kSelectThreads, static_cast<size_t>(nn) * 4, st>>>(scores, nn, N, nn, len, kept, first, moved, 0, nullptr, 0);
-    compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, len, block_B, N, kept, first);
+    compact_kernel<<<dim3(2, U), kCompactThreads, 0, st>>>(kc, vc, nk, nv, len, block_B, N, kept, first, nullptr);
     KD_CUDA(cudaGetLastError());
     return KEYDIFF_OK;
 }

@@ -376,6 +376,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
                 uint4* dk = p.k_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
                 uint4* dv = p.v_cache + (static_cast<size_t>(u) * N + slot) * kRowVec;
                 const uint4 k0 = sk[t], k1 = sk[t + 8], v0 = sv[t], v1 = sv[t + 8];
+                if (!(KD_ROW_OK(slot, N, p.status) && KD_ROW_OK(j, B, p.status))) continue;
                 dk[t] = k0; dk[t + 8] = k1;
                 dv[t] = v0; dv[t + 8] = v1;
                 if (t == 0) {

@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(uint4* k_cache, uint4* v_cache,     // read and written here: no __restrict__
                const uint4* __restrict__ new_k, const uint4* __restrict__ new_v,
                int len, int B, int N, const int32_t* __restrict__ kept_idx,
-               const int32_t* __restrict__ first_evicted) {
+               const int32_t* __restrict__ first_evicted, int32_t* status) {
     __shared__ uint4 stage[kCompactRows * kRowVec];
     const int u = blockIdx.y;
     uint4* cache = blockIdx.x == 0 ? k_cache : v_cache;
@@ -189,7 +189,7 @@ compact_kernel(uint4* k_cache, uint4* v_cache,     // read and written here: no 
         const int cnt = min(kCompactRows, N - base) * kRowVec;
         for (int q = threadIdx.x; q < cnt; q += kCompactThreads) {
             const int src = src_of[base + (q >> 4)];
-            stage[q] = concat_row(cache, block, u, src, len, B, N)[q & 15];
+            stage[q] = KD_ROW_OK(src, len + B, status) ? concat_row(cache, block, u, src, len, B, N)[q & 15] : make_uint4(0, 0, 0, 0);
         }
         __syncthreads();
         uint4* dst = cache + (static_cast<size_t>(u) * N + base) * kRowVec;

@@ -27,8 +27,8 @@ def test_header_symbols_are_exported(lib):
 
 
 def test_strerror_names_every_code(lib):
-    texts = {lib.keydiff_strerror(c).decode() for c in range(0, -7, -1)}
-    assert len(texts) == 7 and "unknown keydiff status" not in texts
+    texts = {lib.keydiff_strerror(c).decode() for c in range(0, -9, -1)}
+    assert len(texts) == 9 and "unknown keydiff status" not in texts
     assert lib.keydiff_strerror(-99).decode() == "unknown keydiff status"
 
 
