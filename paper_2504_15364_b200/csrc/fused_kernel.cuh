@@ -1,34 +1,41 @@
 // Fused path: ONE launch per evicting step.  A thread-block cluster of C CTAs owns one unit
-// (one KV head of one layer of one sequence) from the anchor to the compacted K and V:
+// (one KV head of one layer of one sequence) from the anchor to the compacted K and V, and goes
+// on to the next unit (u + number of clusters) with the next unit's K rows already on their way:
 //
 //   load K      every CTA pulls its contiguous slice of the unit's n key rows on chip exactly
 //               once: most rows into shared memory with TMA bulk copies (cp.async.bulk, one
 //               mbarrier per 16-row tile), the remainder into registers with 128-bit loads.
 //               Nothing is read from HBM twice.
-//   a1 anchor   per-row norm, sum of k/||k|| per CTA; every CTA pushes its 128 partial sums into
-//               all peers' shared memory (DSMEM), one cluster barrier, then each CTA adds the C
-//               partials in rank order (App. B.1, expr. 1).
-//   a2 scores   e_i = -(mu.k_i)/max(||mu|| ||k_i||, eps) from the on-chip rows; the orderable key
-//               of e_i goes into this CTA's part of the key table, the part is then pushed to
-//               all peers with 128-bit DSMEM stores and one cluster barrier completes the table
-//               everywhere (App. B.1, expr. 2).  fp32 scores go to global scratch, coalesced.
-//   a3 select   every CTA selects on its own copy of the table.  Only E = n - N keys go, so the work
-//               is at the low end: a 2048-bin histogram over the unit's own key range, the bin
+//   anchor      (App. B.1, expr. 1)  one-pass steps: the sum of the terms k/||k|| over the cached
+//               rows is carried from step to step (running sum + every CTA's delta of the last
+//               step, folded in double); only the B block rows are normalised, C-th part per CTA,
+//               the shares meet in every CTA's table through DSMEM stores.  Two-pass steps (first
+//               evicting step, after appends, on request) sum all n rows instead.
+//   scores      (App. B.1, expr. 2)  e_i = -(mu.k_i)/max(||mu|| ||k_i||, eps) from the on-chip
+//               rows, norm and dot product in one pass; the orderable key of e_i goes into this
+//               CTA's part of the key table, and the part is pushed to every peer with one bulk
+//               copy each (shared::cluster destination), counted on the peer's own mbarrier: a CTA
+//               selects as soon as ITS table is complete, without a cluster barrier.  fp32 scores
+//               go to global scratch, coalesced.
+//   select      every CTA selects on its own copy of the table.  Only E = n - N keys go, so the
+//               work is at the low end: a 2048-bin histogram over the unit's own key range, the bin
 //               where the running count from below reaches E, a bitmap of the tokens under that
 //               bin, an exact rank among the bin's own few keys.  Crowded bins (many equal scores)
-//               and large units fall back to a histogram over a fixed-point image of e with an
-//               exact rank or a 4x8-bit radix select.  Ties keep the older token (Eq.
-//               efficient-keydiff, topk).
-//   a4 compact  an ordered scan gives every kept row its destination; the rows then leave the
-//               chip tile by tile, and each shared-memory tile is refilled as soon as it has
-//               been written out: K stores hand their tile to the V load of the same rows, V
-//               stores hand it to the K load of the cluster's next unit.  The copy engine's
-//               loads therefore run under the stores (Eq. keydiff, in place, token order).
+//               fall back to a histogram over a fixed-point image of e with an exact rank or a
+//               4x8-bit radix select.  Ties keep the older token (Eq. efficient-keydiff, topk).
+//   compact     prefix counts over the bitmap give every kept row its destination; the rows then
+//               leave the chip tile by tile, and each shared-memory tile is refilled as soon as
+//               it has been written out: K stores hand their tile to the V load of the same rows,
+//               V stores hand it to the K load of the cluster's next unit, which the owning warp
+//               scores while the following tile's stores drain (Eq. keydiff, in place, token
+//               order).  The evicted rows' terms are taken off the running sum on the way out.
 //
-// In-place safety: every K row of the unit is on chip before the first cluster barrier, hence
-// before the first K store.  Every warp arrives at the third cluster barrier only after the V
-// rows it is responsible for have landed (bulk copies waited for, register loads consumed), and
-// no V store is issued before that barrier's wait: every V row that moves is then on chip.
+// Cluster barriers per unit: ONE (before the V stores; two-pass steps have a second, for the anchor's
+// partial sums).  In-place safety: a CTA's K stores start
+// after its key table is complete, i.e. after every peer has scored -- hence holds on chip -- all
+// its K rows of the unit.  Every warp arrives at the cluster barrier only after the V rows it is
+// responsible for have landed (bulk copies waited for, register loads consumed), and no V store is
+// issued before that barrier's wait: every V row that moves is then on chip.
 //
 // No multicast TMA is used anywhere; each CTA issues its own bulk loads.  Every mbarrier wait is
 // bounded: on expiry the kernel records KEYDIFF_ERR_TIMEOUT in the status word and carries on
@@ -52,7 +59,7 @@ constexpr int kCandCap = kFusedThreads;                 // exact-rank stage hand
 constexpr int kMaxCluster = 16;
 constexpr int kFastKeys = 17;                           // fast select: keys per thread held in registers (n <= 8704)
 constexpr int kFastCandCap = 192;                       // fast select: keys of the threshold bin ranked exactly
-constexpr int kReduceBytes = 16 * 1024;   // scratch the dead key table lends: staged row terms (16 KB), quarter sums, lists
+constexpr int kReduceBytes = 16 * 1024;   // least size of the key-table region: while the table is dead it lends two [8][128] double tables
 constexpr int kSmemLimit = 232448;                      // opt-in shared memory per CTA on sm_100
 constexpr int kErrTimeout = -6;                         // KEYDIFF_ERR_TIMEOUT
 constexpr uint32_t kWaitSpins = 1u << 24;               // bound of every mbarrier wait
@@ -109,9 +116,6 @@ __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.w
 __device__ __forceinline__ void cluster_sync_all() { cluster_arrive(); cluster_wait(); }
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
     uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank)); return r;
-}
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 __device__ __forceinline__ void st_cluster_v4(uint32_t addr, const uint4& v) {
     asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
@@ -642,82 +646,7 @@ __device__ __noinline__ void full_select_plan(const uint32_t* keys, int n, int N
 // row that enters the cache adds exactly what it takes away when it is evicted, and no fp32 partial sum of the
 // size of the anchor appears anywhere (an anchor over keys that point in many directions is a cancelling sum;
 // fp32 partial sums would limit it, and with it every score, to about 1e-7 / ||mu||).
-//
-// row_terms: one row group (8 lanes, lane t holding words t and t + 8 of the row) writes the row's 128 terms
-// k_c / max(||k||, eps) -- k_c itself when `raw` -- to out[0..128) in channel order (when `store`).  The whole
-// warp must call (the norm uses the 8-lane butterfly).
-__device__ __forceinline__ void row_terms(const uint4& a, const uint4& b, int t, float inv_eps, bool raw, bool store, float* out) {
-    float2 x[8];
-    unpack_pairs(a, b, x);
-    const float inv = raw ? 1.0f : fminf(approx_rsqrt(pairs_sumsq(x)), inv_eps);
-    if (store) {
-#pragma unroll
-        for (int q = 0; q < 8; q += 2) {
-            // pairs q, q + 1 = four consecutive channels starting at lane_channel(t, 2q)
-            *reinterpret_cast<float4*>(&out[lane_channel(t, 2 * q)]) =
-                make_float4(__fmul_rn(x[q].x, inv), __fmul_rn(x[q].y, inv), __fmul_rn(x[q + 1].x, inv), __fmul_rn(x[q + 1].y, inv));
-        }
-    }
-}
-// terms_sum: staged[j][c] (j < m rows of 128 fp32 terms) summed over j in double; thread (channel c = tid & 127,
-// quarter q = tid >> 7) adds rows q, q + 4, ... in order into acc.  No barrier inside.
-__device__ __forceinline__ void terms_sum(const float* staged, int m, int tid, double& acc) {
-    const int c = tid & (kHeadDim - 1), q = tid >> 7;
-    for (int j = q; j < m; j += 4) acc += static_cast<double>(staged[j * kHeadDim + c]);
-}
-// The four quarters' sums of a channel, in order: returns channel tid's total in threads tid < 128.  part: 4 x 128
-// doubles.  One CTA barrier inside; the caller synchronises before part is reused.
-__device__ __forceinline__ double quarters_sum(double acc, double* part, int tid) {
-    const int c = tid & (kHeadDim - 1), q = tid >> 7;
-    part[q * kHeadDim + c] = acc;
-    __syncthreads();
-    return tid < kHeadDim ? (part[c] + part[kHeadDim + c]) + (part[2 * kHeadDim + c] + part[3 * kHeadDim + c]) : 0.0;
-}
-constexpr int kTermRows = 32;   // rows of terms staged per round (16 KB)
-constexpr int kStashRows = 48;  // evicted cache rows of a slice kept aside as they are (12 KB); at most kGroups
-// Sum of the terms of `count` rows that can be re-read from global memory (row j at row_of(j); the block rows, which
-// nobody writes): phase 1, row group g computes 1/||k|| of rows g, g + 64, ... into inv_sh; phase 2, thread
-// (channel, quarter) re-reads its channel's element of rows q, q + 4, ... and adds the same fp32 products as
-// row_terms forms, in double.  Returns channel tid's sum in threads tid < 128.  All threads call (uniform count);
-// inv_sh: 128 floats, part: 4 x 128 doubles; the caller synchronises before the scratch is reused.
-struct ContiguousRows {   // row j of a run of rows that lie one after the other
-    const uint4* first;
-    __device__ __forceinline__ const uint4* operator()(int j) const { return first + static_cast<size_t>(j) * kRowVec; }
-};
-template <typename RowOf>
-__device__ __forceinline__ double global_rows_terms_sum(RowOf row_of, int count, float inv_eps, bool raw,
-                                                        float* inv_sh, double* part, int tid) {
-    const int g = tid >> 3, t = tid & 7, warp = tid >> 5, c = tid & (kHeadDim - 1), q = tid >> 7;
-    double acc = 0.0;
-    for (int c0 = 0; c0 < count; c0 += kHeadDim) {
-        const int m = min(kHeadDim, count - c0);
-        if (c0 > 0) __syncthreads();   // phase 2 of the previous chunk has read inv_sh
-        for (int j0 = 0; j0 + 4 * warp < m; j0 += kGroups) {   // (warp-uniform bound: pairs_sumsq shuffles)
-            const int j = j0 + g;
-            uint4 a = make_uint4(0, 0, 0, 0), b = a;
-            if (j < m) { const uint4* row = row_of(c0 + j); a = row[t]; b = row[t + 8]; }
-            float2 x[8];
-            unpack_pairs(a, b, x);
-            const float ss = pairs_sumsq(x);
-            if (j < m && t == 0) inv_sh[j] = raw ? 1.0f : fminf(approx_rsqrt(ss), inv_eps);
-        }
-        __syncthreads();
-        for (int jb = q; jb < m; jb += 32) {   // eight rows' elements requested before the first is used
-            uint32_t h[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int j = jb + 4 * i;
-                h[i] = j < m ? __ldg(reinterpret_cast<const uint16_t*>(row_of(c0 + j)) + c) : 0u;
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int j = jb + 4 * i;
-                if (j < m) acc += static_cast<double>(__fmul_rn(__uint_as_float(h[i] << 16), inv_sh[j]));
-            }
-        }
-    }
-    return quarters_sum(acc, part, tid);
-}
+// warp_row_terms (below) forms these terms; both fused kernels and the staged kernels use the same products.
 
 // Evicted tokens before each word of the bitmap: wlocal[w] = number of set bits in words [0, w).  All threads
 // call; uses sel.warp_gt, sel.hist[32..48) and misc[5], misc[6]; ends with a CTA barrier.
