@@ -1059,7 +1059,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         }
         {
             float* sc = p.scores + static_cast<size_t>(u) * p.nmax + seg_a;   // fp32 scores to global scratch, coalesced
-            for (int lr = tid; lr < seg; lr += kFusedThreads) sc[lr] = key_score(keys[seg_a + lr]);
+            for (int lr = tid; lr < seg; lr += kFusedThreads) __stcs(&sc[lr], key_score(keys[seg_a + lr]));
             for (int b = tid; b < kBins; b += kFusedThreads) hist[b] = 0;
             for (int wd = tid; wd < nwords; wd += kFusedThreads) bitmap[wd] = 0;
             if (tid == 0) { misc[0] = 0; misc[1] = n; }
@@ -1105,7 +1105,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         for (int lr = tid; lr < seg; lr += kFusedThreads) {   // kept-index list, coalesced (destinations ascend with lr)
             const int d = dst_of[lr];
             if (d >= 0) {
-                p.kept_idx[static_cast<size_t>(u) * N + d] = seg_a + lr;
+                __stcs(&p.kept_idx[static_cast<size_t>(u) * N + d], seg_a + lr);
                 if (p.kept_mirror) p.kept_mirror[static_cast<size_t>(u) * N + d] = seg_a + lr;
             }
         }
