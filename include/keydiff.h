@@ -160,7 +160,9 @@ KEYDIFF_API int keydiff_create(const keydiff_config* cfg, keydiff_ctx** out);
  * kernels return normally; the call itself has returned KEYDIFF_OK long before.  A non-zero
  * status word means that the cache rows, scores and lists of that step (and of every later
  * step of the ctx: the word is never cleared) are unspecified; restore the caches from a
- * copy and use a new ctx (keydiff_set_len / keydiff_set_positions).  Non-finite keys give an
+ * copy and use a new ctx (keydiff_set_len / keydiff_set_positions).  (With slot reuse a thread block whose own
+ * wait expired places no further rows; the ordered kernel carries on to its normal end -- a check in its store
+ * loops was measured at 3-5 % of the step -- so rows that never arrived on chip may be stored.)  Non-finite keys give an
  * unspecified selection, never a fault.
  */
 KEYDIFF_API int keydiff_evict(keydiff_ctx* ctx, void* k_cache, void* v_cache,

@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
     int* blk_of = slot_of + p.max_block;                   // kept block rows, ascending
     SelectSmem& sel = *reinterpret_cast<SelectSmem*>(smem + L.sel);
     float* mu_sh = reinterpret_cast<float*>(smem + L.mu);
-    int* misc = reinterpret_cast<int*>(smem + L.misc);   // 0 ncand, 1 first evicted, 2 need_eq, 3 threshold key, 5/6 prefix carry
+    int* misc = reinterpret_cast<int*>(smem + L.misc);   // 0 ncand, 1 first evicted, 2 need_eq, 3 threshold key, 5/6 prefix carry, 12 a wait ran out
     const uint32_t ring_sa = smem_addr(ring), mbar_sa = smem_addr(smem + L.mbar), keys_sa = smem_addr(keys);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = tid >> 3, t = tid & 7, sub = lane >> 3;
@@ -121,6 +121,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
     if (tid == 0) {
         for (int j = 0; j < p.ring_tiles; ++j) mbar_init(mbar_sa + 8 * j, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        misc[12] = 0;
     }
     __syncthreads();
     if (p.stagger_ns != 0 && cluster_id != 0) {   // bounded start-up delay that spreads the clusters' phases
@@ -209,7 +210,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
 #pragma unroll 1
             for (int j = 0; j < cnt_w; ++j) {
                 const int phys = warp + kFusedWarps * c_d;
-                mbar_wait(mbar_sa + 8 * phys, (c_par >> c_d) & 1u, p.status);
+                // (a tile that never landed: from then on this CTA places no row and reports no change to the running sum)
+                if (!mbar_wait(mbar_sa + 8 * phys, (c_par >> c_d) & 1u, p.status)) misc[12] = 1;
                 c_par ^= 1u << c_d;
                 const int lo = (warp + kFusedWarps * j) * kTileRows;   // first slice row of the tile
                 const uint4* tile = ring + phys * kTileRows * kRowVec;
@@ -363,13 +365,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) slot_evict_kernel(const Slot
                 }
                 const double gone = cta_sum_of_warp_sums(acc, reinterpret_cast<double*>(keys), tid);   // the key table is dead until the next unit
                 if (tid < kHeadDim)
-                    p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (crank == 0 ? block_sum : 0.0) - gone;
+                    p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = misc[12] == 0 ? (crank == 0 ? block_sum : 0.0) - gone : 0.0;
                 // (the barriers inside the sum lie behind every read of an evicted row: its slot may be overwritten)
             }
             // (b) kept block row r into freed slot r.  For r < evicted_cache that slot is evicted row r, which this
             // same CTA re-read in (a), in front of the barrier above.
 #pragma unroll 2
-            for (int r = r_first; r < kb; r += stride) {
+            for (int r = misc[12] == 0 ? r_first : kb; r < kb; r += stride) {
                 const int slot = slot_of[r], j = blk_of[r];
                 const uint4* sk = p.new_k + (static_cast<size_t>(u) * B + j) * kRowVec;
                 const uint4* sv = p.new_v + (static_cast<size_t>(u) * B + j) * kRowVec;
