@@ -761,7 +761,6 @@ __device__ __forceinline__ double cta_sum_of_warp_sums(const double (&acc)[4], d
     }
     return s;
 }
-constexpr int kPreRows = 4;   // block rows per warp and kind requested before the K stores (the rest after them)
 
 // kRegRows = rows per row group that live in registers (the host picks the smallest instance that
 // holds a slice together with the shared-memory rows).
@@ -777,7 +776,11 @@ constexpr int kPreRows = 4;   // block rows per warp and kind requested before t
 // the next step folds the deltas into the running sum, in double precision and in a fixed order.
 // kOnePass = false recomputes the anchor from all n rows (first evicting step, after set_len / reset / appends,
 // and periodically).
-template <int kRegRows, bool kOnePass>
+//
+// kPreRows: block rows per warp and kind that are requested before the K stores and held in registers across them
+// (the rest is read after the stores, latency exposed).  The host picks 1 when a CTA's share of the block is at
+// most one row per warp (B <= 16 C) -- the registers this frees shorten the store loop -- and 4 otherwise.
+template <int kRegRows, bool kOnePass, int kPreRows>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const FusedParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int C = p.cluster;

@@ -130,18 +130,20 @@ inline bool slot_reuse(const keydiff_ctx* c) { return c->cfg.compaction == KEYDI
 using FusedKernel = void (*)(kd::FusedParams);
 
 // Kernel instance for `reg_rows` register-resident rows per row group (rounded up to one that is
-// built); one_pass = the variant that takes the anchor from the running sum.
-template <bool kOnePass>
+// built); one_pass = the variant that takes the anchor from the running sum; few_pre = the variant that holds one
+// block row per warp and kind across the K stores instead of four (one-pass kernels only).
+template <bool kOnePass, int kPre>
 FusedKernel fused_instance_of(int reg_rows, int* built) {
     using namespace kd;
-    if (reg_rows <= 0) { *built = 0; return fused_evict_kernel<0, kOnePass>; }
-    if (reg_rows <= 2) { *built = 2; return fused_evict_kernel<2, kOnePass>; }
-    if (reg_rows <= 4) { *built = 4; return fused_evict_kernel<4, kOnePass>; }
-    if (reg_rows <= 5) { *built = 5; return fused_evict_kernel<5, kOnePass>; }
-    *built = 6; return fused_evict_kernel<6, kOnePass>;
+    if (reg_rows <= 0) { *built = 0; return fused_evict_kernel<0, kOnePass, kPre>; }
+    if (reg_rows <= 2) { *built = 2; return fused_evict_kernel<2, kOnePass, kPre>; }
+    if (reg_rows <= 4) { *built = 4; return fused_evict_kernel<4, kOnePass, kPre>; }
+    if (reg_rows <= 5) { *built = 5; return fused_evict_kernel<5, kOnePass, kPre>; }
+    *built = 6; return fused_evict_kernel<6, kOnePass, kPre>;
 }
-FusedKernel fused_instance(int reg_rows, int* built, bool one_pass = false) {
-    return one_pass ? fused_instance_of<true>(reg_rows, built) : fused_instance_of<false>(reg_rows, built);
+FusedKernel fused_instance(int reg_rows, int* built, bool one_pass = false, bool few_pre = false) {
+    if (!one_pass) return fused_instance_of<false, 4>(reg_rows, built);
+    return few_pre ? fused_instance_of<true, 1>(reg_rows, built) : fused_instance_of<true, 4>(reg_rows, built);
 }
 
 // Co-resident clusters of `C` CTAs of the kernel `kern` with `smem` bytes each.
@@ -201,7 +203,8 @@ bool plan_fused(keydiff_ctx* c, int sm_count) {
     // the attributes of the chosen instance (the loop may have left another size's values behind)
     int built = 0;
     return max_active_clusters(fused_instance(c->fused_reg_rows, &built, false), c->cluster, c->fused_smem_bytes, sm_count) >= 1 &&
-           max_active_clusters(fused_instance(c->fused_reg_rows, &built, true), c->cluster, c->fused_smem_bytes, sm_count) >= 1;
+           max_active_clusters(fused_instance(c->fused_reg_rows, &built, true, false), c->cluster, c->fused_smem_bytes, sm_count) >= 1 &&
+           max_active_clusters(fused_instance(c->fused_reg_rows, &built, true, true), c->cluster, c->fused_smem_bytes, sm_count) >= 1;
 }
 
 // Slot reuse: cluster size and ring of the streaming kernel for units of up to nmax rows; false if it
@@ -350,7 +353,8 @@ int launch_fused(keydiff_ctx* c, uint4* kc, uint4* vc, const uint4* nk, const ui
     attr[0].val.clusterDim.x = c->cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     int built = 0;
-    KD_CUDA(cudaLaunchKernelEx(&cfg, fused_instance(c->fused_reg_rows, &built, one_pass), p));
+    const bool few_pre = B <= 16 * c->cluster;   // a CTA's share of the block: at most one row per warp
+    KD_CUDA(cudaLaunchKernelEx(&cfg, fused_instance(c->fused_reg_rows, &built, one_pass, few_pre), p));
     c->anchor_par ^= 1;
     c->anchor_valid = true;
     c->steps_since_full = one_pass ? c->steps_since_full + 1 : 0;
