@@ -867,7 +867,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
     // barrier every CTA adds the C shares in rank order to the folded running sum: the same anchor bits everywhere.
     const int b_per = (B + C - 1) / C;
     const int b_lo = min(B, crank * b_per), b_hi = min(B, b_lo + b_per);
-    double my_share = 0.0;       // tid < 128: channel tid of this CTA's share of this unit's block sum
+    // (this CTA's own share of a unit's block sum is not kept in a register: every CTA pushes its share to all CTAs
+    // of the cluster, itself included, so it stays readable in row `crank` of this CTA's own table until the next push)
     bool tiles_scored = false;   // this unit's tiles were scored behind the previous unit's V rows
     int cur = 0;                 // which of the two anchor buffers holds this unit's anchor
     auto fold_running_sum = [&](int uu) -> double {   // threads tid < 128
@@ -898,10 +899,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
             const uint4* blk = p.new_k + static_cast<size_t>(cluster_id) * B * kRowVec;
             for (int j = b_lo + warp; j < b_hi; j += kFusedWarps)   // (warp-uniform)
                 warp_row_terms(reinterpret_cast<const uint2*>(blk + static_cast<size_t>(j) * kRowVec)[lane], true, inv_eps, raw, acc);
-            my_share = cta_sum_of_warp_sums(acc, gone_tab, tid);   // (nobody uses the key table before the first unit's scores)
+            const double first_share = cta_sum_of_warp_sums(acc, gone_tab, tid);   // (nobody uses the key table before the first unit's scores)
             __syncthreads();   // the table is free again before any key is written
+            if (tid < kHeadDim) push_share(first_share);
         }
-        if (tid < kHeadDim) push_share(my_share);
         cluster_sync_all();
         if (tid < kHeadDim) anchor_from_shares(folded, mu_buf);
         __syncthreads();
@@ -1194,7 +1195,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         KD_STAMP(6);
         // ------------------------------------------------------------ the block rows of this CTA's range (requested before the
         // stores), every warp's sums into the tables, one barrier, and the delta and the next share are complete
-        double share_next = 0.0;
         {
 #pragma unroll
             for (int k = 0; k < kPreRows; ++k) {
@@ -1229,10 +1229,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
                 double gsum = 0.0, nsum = 0.0;
 #pragma unroll
                 for (int w = 0; w < 8; ++w) { gsum += gone_tab[w * kHeadDim + tid]; nsum += next_tab[w * kHeadDim + tid]; }
-                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass ? my_share : 0.0) - gsum;
+                p.anchor_delta[(static_cast<size_t>(u) * C + crank) * kHeadDim + tid] = (kOnePass ? partials[crank * kHeadDim + tid] : 0.0) - gsum;
                 if (next_share) {
-                    share_next = nsum;
-                    push_share(share_next);   // read by every CTA after the third cluster barrier
+                    push_share(nsum);   // read by every CTA after the third cluster barrier (and by this one as its own share, a unit later)
                 }
             }
         }
@@ -1321,7 +1320,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_evict_kernel(const Fus
         if (kOnePass && un < p.U) {
             tiles_scored = true;
             cur ^= 1;
-            my_share = share_next;
         }
         KD_STAMP(11);
         __syncthreads();   // dst_of is free for the next unit
