@@ -74,15 +74,17 @@ __host__ __device__ inline FusedLayout fused_layout(int smem_rows, int nkeys, in
     FusedLayout L;
     int off = 0;
     auto take = [&off](int bytes) { const int o = off; off += (bytes + 127) & ~127; return o; };
+    // the regions whose size does not depend on the launch come first: their addresses are compile-time constants, which
+    // keeps them out of the registers
+    L.misc = take(128);
+    L.mbar = take((kMaxTiles + 1) * 8);   // one per tile + the key exchange's
+    L.mu = take(2 * kHeadDim * 4);   // this unit's anchor and the next unit's
+    L.sel = take(static_cast<int>(sizeof(SelectSmem)));
+    L.work = take(kBins * 4);   // warp-reduction scratch / histogram / destination table (never live together)
     L.rows = take(smem_rows * kRowBytes);
     L.keys = take(nkeys * 4 > kReduceBytes ? nkeys * 4 : kReduceBytes);   // also the reduction scratch while the table is dead
-    L.work = take(kBins * 4);   // warp-reduction scratch / histogram / destination table (never live together)
     L.xchg = take(2 * kCandCap * 4 + C * kHeadDim * 8);   // candidates of the threshold bin | [C][128] doubles pushed by the peers
     L.bitmap = take(2 * ((nkeys + 31) / 32) * 4);   // evicted-token bitmap, evicted-before count of every word
-    L.sel = take(static_cast<int>(sizeof(SelectSmem)));
-    L.mu = take(2 * kHeadDim * 4);   // this unit's anchor and the next unit's
-    L.mbar = take((kMaxTiles + 1) * 8);   // one per tile + the key exchange's
-    L.misc = take(128);
     L.total = off;
     return L;
 }
