@@ -25,6 +25,7 @@
 
 namespace kd {
 
+constexpr int kSlotMaxRing = 3 * kFusedWarps;   // at most three tiles per warp in the ring
 constexpr int kSlotMaxBlock = 1024;   // the three lists of a step live in shared memory, max_block entries each
 
 struct SlotLayout {
@@ -34,16 +35,17 @@ __host__ __device__ inline SlotLayout slot_layout(int ring_tiles, int nkeys, int
     SlotLayout L;
     int off = 0;
     auto take = [&off](int bytes) { const int o = off; off += (bytes + 127) & ~127; return o; };
+    // fixed-size regions first: compile-time addresses (the ring's too), which keeps them out of the registers
+    L.misc = take(128);
+    L.mbar = take(kSlotMaxRing * 8);
+    L.mu = take(kHeadDim * 4);
+    L.sel = take(static_cast<int>(sizeof(SelectSmem)));
+    L.cand = take(2 * kCandCap * 4);     // keys and indices of the threshold bin
+    L.work = take(kBins * 4);            // warp-reduction scratch / histogram
     L.ring = take(ring_tiles * kTileRows * kRowBytes);
     L.keys = take(nkeys * 4 > kReduceBytes ? nkeys * 4 : kReduceBytes);   // also the reduction scratch while the table is dead
-    L.work = take(kBins * 4);            // warp-reduction scratch / histogram
     L.bitmap = take(2 * nwords * 4);     // evicted-candidate bitmap, evicted-before count of every word
-    L.cand = take(2 * kCandCap * 4);     // keys and indices of the threshold bin
     L.lists = take(3 * max_block * 4);   // evicted candidates, freed slots, kept block rows
-    L.sel = take(static_cast<int>(sizeof(SelectSmem)));
-    L.mu = take(kHeadDim * 4);
-    L.mbar = take(ring_tiles * 8);
-    L.misc = take(128);
     L.total = off;
     return L;
 }
