@@ -37,8 +37,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (bytes per step of the named workload); None = not captured.
-NCU_TRAFFIC_BYTES = {("llama31_8b_n8192", "ordered"): 2.1161e9, ("llama31_8b_n8192", "slot_reuse"): 5.947e8,
-                     ("llama32_3b_n2048", "ordered"): 4.273e8, ("llama32_3b_n2048", "slot_reuse"): 1.363e8}
+NCU_TRAFFIC_BYTES = {("llama31_8b_n8192", "ordered"): 2.1161e9, ("llama31_8b_n8192", "slot_reuse"): 5.955e8,
+                     ("llama32_3b_n2048", "ordered"): 4.287e8, ("llama32_3b_n2048", "slot_reuse"): 1.360e8}
 
 
 def measured_peak():
