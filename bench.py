@@ -247,6 +247,8 @@ def run_ours(args):
     wl = synth.WORKLOADS[args.workload]
     if args.batch > 0:
         wl = synth.scaled(wl, batch=args.batch)
+    if args.block > 0:
+        wl = synth.scaled(wl, block=args.block)
     U, N, B, d = wl.units, wl.budget, wl.block, wl.head_dim
     path = {"auto": binding.KEYDIFF_PATH_AUTO, "staged": binding.KEYDIFF_PATH_STAGED,
             "fused": binding.KEYDIFF_PATH_FUSED}[args.path]
@@ -396,6 +398,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0,
                     help="run the workload at this batch size instead of its own (profiling aid: the decode workload's unit shape "
                          "at batch 2 is 2 GB instead of 34 GB); the line's config says so")
+    ap.add_argument("--block", type=int, default=0,
+                    help="run the workload with another block size B (0 = the workload's own), e.g. 1 for token-by-token decode")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -106,3 +106,17 @@ def test_clustered_keys_300_steps_keep_the_plain_relative_bound(compaction):
     worst = stream_and_check(wl, compaction, 300, steps, list(range(wl.units)))
     assert worst["checked"] == len(steps)
     assert worst["plain_rel"] < 1e-5 and worst["err_over_tol"] < 0.5, worst
+
+
+@pytest.mark.parametrize("compaction", LAYOUTS)
+def test_token_by_token_decode_at_the_full_budget(compaction):
+    # The decode cadence of Eq. block_processing with B = 1 (Sec. 2.4: one token appended, one evicted) at the decode
+    # workload's full unit shape (N = 8192, 256 units = batch 1): the cache is filled token by token through the
+    # library, then 200 single-token steps evict, on the running anchor.
+    wl = synth.scaled(synth.WORKLOADS["decode_b32_n8192"], batch=1, block=1, total_tokens=8192 + 200)
+    assert wl.evict_steps == 200 and wl.fill_steps == 8192
+    steps = {0, 1, 2, 50, 100, 199}
+    units = sorted(set(np.linspace(0, wl.units - 1, 4).astype(int).tolist()))
+    worst = stream_and_check(wl, compaction, 200, steps, units)
+    assert worst["checked"] == len(steps)
+    assert worst["err_over_tol"] < 0.5 and worst["plain_rel"] < 5e-6, worst
